@@ -1,0 +1,352 @@
+"""CPU oracle for the CriticalKV prefill-time compression step.
+
+TEST INFRASTRUCTURE ONLY.  This file is a slow, plain NumPy restatement of the
+method of "Optimizing KV Cache Eviction from an Output Perturbation
+Perspective" (Algorithm 1, Algorithm 2, Eq. 2, Theorems 3.2 / 3.3 / 3.5 and the
+relaxed-bound theorem of the appendix).  It exists to check the CUDA library;
+it shares no code with it and nothing in the product path may import it.
+
+Every floating-point quantity is computed in float64 from the stored inputs
+widened exactly, with one exception that is part of the contract with the CUDA
+path: the arithmetic that *decides integers* (group reduction of the scores and
+everything downstream: budgets, the two top-k stages) runs in IEEE float32 in a
+fixed operation order, because that is the precision the kernels decide in.
+
+Pins (tests/test_oracle_*.py): softmax rows sum to one; w = 1, kp = 1 reduces
+to a library softmax; max-pool against a library sliding maximum and a loop;
+the projection norm against closed forms (identity / one-hot / scaled rows) and
+a triple loop; Theorem 3.2 as an identity; Theorem 3.3 by enumerating every
+subset on n <= 16; Theorem 3.5's arg-min by enumerating every stage-2
+completion; alpha = 1 and constant-norm special cases; tie-breaking and budget
+invariants.  The whole-path output on the large synthetic configurations has no
+printed worked example in the paper to compare with: beyond those pins it is
+"parity unpinned".
+
+Readings of the paper where it is silent or inconsistent (each is an argument,
+defaults below): logit scale 1/sqrt(head_dim) (Eq. 2); causal mask inside the
+window; both stages use the pooled window mean (Algorithm 2 hands its
+accumulated weights to Algorithm 1); GQA groups reduce by the arithmetic mean
+of the per-query-head scores; b' = floor(alpha * b); ties go to the lower
+index; retained rows keep their original order.
+"""
+from __future__ import annotations
+
+import math
+from itertools import combinations
+
+import numpy as np
+
+F64 = np.float64
+F32 = np.float32
+
+
+# ----------------------------------------------------------------------------
+# Step 1: observation-window attention (Algorithm 2, steps "Q_hat = Q[-n':]",
+# "A = softmax(Q_hat K^T); A_bar = A.mean(dim=0)", "A_bar = maxpooling(A_bar)";
+# Eq. 2 for the softmax and its scale)
+# ----------------------------------------------------------------------------
+def window_softmax(Qw_h, K_g, scale):
+    """Causal softmax of the w window queries of one query head over all n keys.
+
+    Window row j sits at sequence position n - w + j and sees keys i <= n - w + j.
+    Returns A [w, n] float64, rows summing to one, masked entries exactly 0.
+    """
+    Qw_h = np.asarray(Qw_h, dtype=F64)
+    K_g = np.asarray(K_g, dtype=F64)
+    w, n = Qw_h.shape[0], K_g.shape[0]
+    logits = (Qw_h @ K_g.T) * F64(scale)
+    pos = n - w + np.arange(w)
+    visible = np.arange(n)[None, :] <= pos[:, None]
+    logits = np.where(visible, logits, -np.inf)
+    m = logits.max(axis=1, keepdims=True)
+    e = np.exp(logits - m)
+    e[~visible] = 0.0
+    return e / e.sum(axis=1, keepdims=True)
+
+
+def window_mean(A):
+    """A_bar[i] = (1/w) sum_j A[j, i]  (Algorithm 2: A.mean(dim=0))."""
+    A = np.asarray(A, dtype=F64)
+    return A.sum(axis=0) / F64(A.shape[0])
+
+
+def max_pool(x, kp):
+    """Stride-1 max-pool along the sequence, window kp centred on i, clipped
+    at both borders, output length n (Algorithm 2: maxpooling; kernel size
+    from Section 4.1)."""
+    if kp < 1 or kp % 2 == 0:
+        raise ValueError("pool kernel must be odd and >= 1")
+    x = np.asarray(x)
+    n = x.shape[-1]
+    r = (kp - 1) // 2
+    out = x.copy()
+    for d in range(1, r + 1):
+        # neighbour at i + d
+        out[..., : n - d] = np.maximum(out[..., : n - d], x[..., d:])
+        # neighbour at i - d
+        out[..., d:] = np.maximum(out[..., d:], x[..., : n - d])
+    return out
+
+
+def pooled_window_attention(Qw, K, kp, scale=None):
+    """P [Hq, n] float64: per query head, max-pooled window-mean attention.
+
+    Qw [Hq, w, dh], K [Hkv, n, dh]; query head h reads KV head h // G.
+    """
+    Hq, w, dh = Qw.shape
+    Hkv, n, _ = K.shape
+    G = Hq // Hkv
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(dh)
+    P = np.empty((Hq, n), dtype=F64)
+    for h in range(Hq):
+        A = window_softmax(Qw[h], K[h // G], scale)
+        P[h] = max_pool(window_mean(A), kp)
+    return P
+
+
+# ----------------------------------------------------------------------------
+# Step 2: projected value-row norm (Algorithm 1: "V_cal = V W^O" and the
+# "L1 norm of each row"; Theorem 3.3 for the role of the norm)
+# ----------------------------------------------------------------------------
+def projection_norm(V, WO, *, rows=None, chunk=2048, norm="l1"):
+    """nu [Hq, n] float64 with nu[h, i] = || V[h // G, i, :] @ WO[h] ||_1.
+
+    V [Hkv, n, dh]; WO [Hq, dh, dm] (head h's rows of the output projection).
+    The product is materialised chunk by chunk and reduced row-wise.
+    ``rows``: optional index array: only these token rows are computed
+    (result [Hq, len(rows)]).
+    """
+    Hkv, n, dh = V.shape
+    Hq, _, dm = WO.shape
+    G = Hq // Hkv
+    sel = np.arange(n) if rows is None else np.asarray(rows)
+    nu = np.empty((Hq, sel.size), dtype=F64)
+    for h in range(Hq):
+        W = np.asarray(WO[h], dtype=F64)
+        Vg = V[h // G]
+        for s in range(0, sel.size, chunk):
+            r = sel[s:s + chunk]
+            proj = np.asarray(Vg[r], dtype=F64) @ W          # [rows, dm]
+            if norm == "l1":
+                nu[h, s:s + chunk] = np.abs(proj).sum(axis=1)
+            elif norm == "l2":
+                nu[h, s:s + chunk] = np.sqrt((proj * proj).sum(axis=1))
+            else:
+                raise ValueError(norm)
+    return nu
+
+
+# ----------------------------------------------------------------------------
+# Step 3: scores per KV head and budgets
+# (Algorithm 1: "A_cal = (A + eps) * row norms", "b' = b x alpha; b'' = b - b'";
+#  Algorithm 2: "allocate budget b across heads")
+# Decision arithmetic: IEEE float32, fixed order (see module docstring).
+# ----------------------------------------------------------------------------
+def group_scores(P, nu, G, eps=1e-4):
+    """a [Hkv, n], c [Hkv, n] float32.
+
+    a_g = (P_{gG} + P_{gG+1} + ... ) / G                  (left-to-right float32 sums)
+    c_g = ((P_{gG}+eps)*nu_{gG} + (P_{gG+1}+eps)*nu_{gG+1} + ...) / G
+    every +, * and / a separately rounded float32 operation.
+    """
+    P = np.asarray(P).astype(F32)
+    nu = np.asarray(nu).astype(F32)
+    Hq, n = P.shape
+    Hkv = Hq // G
+    e = F32(eps)
+    Gf = F32(G)
+    a = np.empty((Hkv, n), dtype=F32)
+    c = np.empty((Hkv, n), dtype=F32)
+    for g in range(Hkv):
+        sa = P[g * G].copy()
+        sc = ((P[g * G] + e).astype(F32) * nu[g * G]).astype(F32)
+        for h in range(g * G + 1, (g + 1) * G):
+            sa = (sa + P[h]).astype(F32)
+            t = ((P[h] + e).astype(F32) * nu[h]).astype(F32)
+            sc = (sc + t).astype(F32)
+        a[g] = (sa / Gf).astype(F32)
+        c[g] = (sc / Gf).astype(F32)
+    return a, c
+
+
+def split_budget(b, alpha):
+    """b' = floor(alpha * b) in double precision, b'' = b - b' (Algorithm 1)."""
+    b1 = int(math.floor(float(F32(alpha)) * float(b)))
+    b1 = min(max(b1, 0), int(b))
+    return b1, int(b) - b1
+
+
+def stable_topk(x, k):
+    """Indices of the k largest entries; equal values go to the lower index.
+    Returned in rank order (best first)."""
+    x = np.asarray(x)
+    if k <= 0:
+        return np.empty(0, dtype=np.int64)
+    order = np.argsort(-x, kind="stable")
+    return order[:k]
+
+
+def allocate_budgets(a, mode, budget):
+    """Per-KV-head budgets b_g (Algorithm 2, budget allocation step).
+
+    uniform : every head gets ``budget``.
+    adaptive: the ``budget`` largest entries of the flattened [Hkv * n]
+              attention scores are counted per head (ties: lower flattened
+              index g * n + i first).
+    """
+    Hkv, n = a.shape
+    if mode == "uniform":
+        return np.full(Hkv, int(budget), dtype=np.int64)
+    if mode == "adaptive":
+        top = stable_topk(a.reshape(-1), int(budget))
+        return np.bincount(top // n, minlength=Hkv).astype(np.int64)
+    raise ValueError(mode)
+
+
+# ----------------------------------------------------------------------------
+# Step 4: two-stage selection of one head (Algorithm 1, stage 1 and stage 2)
+# ----------------------------------------------------------------------------
+def two_stage_select(a_g, c_g, b, alpha):
+    """Returns (S1, S2): stage-1 indices = top-b' of a_g; stage-2 indices =
+    top-b'' of c_g among the entries stage 1 left.  Both ascending."""
+    n = a_g.shape[0]
+    b1, b2 = split_budget(b, alpha)
+    S1 = stable_topk(a_g, b1)
+    rest = np.ones(n, dtype=bool)
+    rest[S1] = False
+    cand = np.nonzero(rest)[0]                      # ascending, so ties keep index order
+    S2 = cand[stable_topk(np.asarray(c_g)[cand], b2)]
+    return np.sort(S1), np.sort(S2)
+
+
+def select(P, nu, *, G, budget_mode, budget, alpha=0.5, eps=1e-4, budgets_in=None):
+    """Steps 3+4 for one layer.
+
+    Returns dict(idx [Btot] int32 packed by head, ascending inside a head;
+    offsets [Hkv+1] int32; stage [Btot] uint8 (1 or 2); a, c float32; budgets).
+    """
+    a, c = group_scores(P, nu, G, eps)
+    Hkv, n = a.shape
+    if budget_mode == "given":
+        budgets = np.asarray(budgets_in, dtype=np.int64)
+    else:
+        budgets = allocate_budgets(a, budget_mode, budget)
+    idx, stage, offsets = [], [], [0]
+    for g in range(Hkv):
+        S1, S2 = two_stage_select(a[g], c[g], int(budgets[g]), alpha)
+        S = np.concatenate([S1, S2])
+        st = np.concatenate([np.ones(S1.size, np.uint8), np.full(S2.size, 2, np.uint8)])
+        order = np.argsort(S, kind="stable")
+        idx.append(S[order])
+        stage.append(st[order])
+        offsets.append(offsets[-1] + S.size)
+    return dict(idx=np.concatenate(idx).astype(np.int32), stage=np.concatenate(stage),
+                offsets=np.asarray(offsets, dtype=np.int32), a=a, c=c, budgets=budgets)
+
+
+# ----------------------------------------------------------------------------
+# Step 5: compaction (Algorithm 1: "add K_i, V_i to K_hat, V_hat")
+# ----------------------------------------------------------------------------
+def compact(K_store, V_store, idx, offsets):
+    """Row gather of the stored (unwidened) K, V: [Btot, dh] each, packed like idx."""
+    Hkv = K_store.shape[0]
+    Ko = np.empty((idx.size, K_store.shape[2]), dtype=K_store.dtype)
+    Vo = np.empty_like(Ko)
+    for g in range(Hkv):
+        s, e = int(offsets[g]), int(offsets[g + 1])
+        Ko[s:e] = K_store[g][idx[s:e]]
+        Vo[s:e] = V_store[g][idx[s:e]]
+    return Ko, Vo
+
+
+def compress_layer(Qw, K, V, WO, *, kp, budget_mode, budget, alpha=0.5, eps=1e-4, scale=None,
+                   K_store=None, V_store=None):
+    """The whole path for one layer, step by step."""
+    G = Qw.shape[0] // K.shape[0]
+    P = pooled_window_attention(Qw, K, kp, scale)
+    nu = projection_norm(V, WO)
+    out = select(P, nu, G=G, budget_mode=budget_mode, budget=budget, alpha=alpha, eps=eps)
+    Ko, Vo = compact(K if K_store is None else K_store, V if V_store is None else V_store,
+                     out["idx"], out["offsets"])
+    out.update(P=P, nu=nu, K_hat=Ko, V_hat=Vo)
+    return out
+
+
+# ----------------------------------------------------------------------------
+# Diagnostics: the quantities of Section 3 (Definition 3.1, Theorems 3.2, 3.3,
+# 3.5, Assumption 3.4, relaxed bound).  Single query row, single head.
+# ----------------------------------------------------------------------------
+def masked_softmax(logits, keep):
+    """A' = softmax(M + logits), M_i = -inf for evicted entries (Section 3.3)."""
+    logits = np.asarray(logits, dtype=F64)
+    keep = np.asarray(keep, dtype=bool)
+    z = np.where(keep, logits, -np.inf)
+    m = z.max()
+    e = np.where(keep, np.exp(z - m), 0.0)
+    return e / e.sum()
+
+
+def perturbation(A, A_prime, Vproj):
+    """L = || (A - A') V W^O ||_1 (Definition 3.1 / Section 3.3)."""
+    return float(np.abs((np.asarray(A, F64) - np.asarray(A_prime, F64)) @ np.asarray(Vproj, F64)).sum())
+
+
+def theta_bound(A, nu, keep):
+    """theta of Theorem 3.3."""
+    A, nu = np.asarray(A, F64), np.asarray(nu, F64)
+    keep = np.asarray(keep, dtype=bool)
+    C = float((A * nu).sum())
+    mass = float(A[keep].sum())
+    return C - (2.0 - 1.0 / mass) * float((A[keep] * nu[keep]).sum())
+
+
+def theta_hat_bound(A, nu, keep1, keep2):
+    """theta_hat of Theorem 3.5 (sigma = attention mass of the stage-1 set)."""
+    A, nu = np.asarray(A, F64), np.asarray(nu, F64)
+    k1, k2 = np.asarray(keep1, bool), np.asarray(keep2, bool)
+    sigma = float(A[k1].sum())
+    C = float((A * nu).sum())
+    f = 2.0 - 1.0 / sigma
+    return C - f * float((A[k1] * nu[k1]).sum()) - f * float((A[k2] * nu[k2]).sum())
+
+
+def theta_relax_bound(A, nu, keep1, keep2):
+    """theta_hat^relax of the appendix theorem (M = min_i nu_i)."""
+    A, nu = np.asarray(A, F64), np.asarray(nu, F64)
+    k1, k2 = np.asarray(keep1, bool), np.asarray(keep2, bool)
+    sigma = float(A[k1].sum())
+    C = float((A * nu).sum())
+    f = 2.0 - 1.0 / sigma
+    return C - f * float((A[k1] * nu[k1]).sum()) - float(nu.min()) * f * float(A[k2].sum())
+
+
+def stage1_mass(a_g, b, alpha):
+    """sigma of Assumption 3.4: attention collected by stage 1."""
+    b1, _ = split_budget(b, alpha)
+    return float(np.sort(np.asarray(a_g, F64))[::-1][:b1].sum())
+
+
+def post_eviction_output(Qw_h, K_g, V_g, keep_idx, scale):
+    """o_hat [w, dh]: window queries attending only to the retained entries
+    (causal by original position), before W^O.  ``keep_idx=None`` = full cache."""
+    Qw_h, K_g, V_g = (np.asarray(x, dtype=F64) for x in (Qw_h, K_g, V_g))
+    w, n = Qw_h.shape[0], K_g.shape[0]
+    keep = np.ones(n, bool) if keep_idx is None else np.isin(np.arange(n), keep_idx)
+    logits = (Qw_h @ K_g.T) * F64(scale)
+    pos = n - w + np.arange(w)
+    out = np.zeros((w, V_g.shape[1]), dtype=F64)
+    for j in range(w):
+        vis = keep & (np.arange(n) <= pos[j])
+        if not vis.any():
+            continue
+        out[j] = masked_softmax(logits[j], vis) @ V_g
+    return out
+
+
+def all_subsets(n, b):
+    """Every subset of size b as a boolean mask (tiny n only)."""
+    for comb in combinations(range(n), b):
+        m = np.zeros(n, dtype=bool)
+        m[list(comb)] = True
+        yield m
