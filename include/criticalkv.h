@@ -1,0 +1,153 @@
+/*
+ * criticalkv.h -- C ABI of the CriticalKV prefill-time KV-cache compression step for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one layer-level operation of "Optimizing KV Cache Eviction from an Output Perturbation
+ * Perspective": score every cached KV entry of every head, keep a budgeted subset with the paper's two-stage
+ * perturbation-constrained rule, and compact K/V.  The three entry points follow the paper's problem statement
+ * (Algorithm 1 inputs: budget b, query state, K, V, W^O, alpha; Algorithm 2 inputs: Q, K, V, window size):
+ *
+ *   criticalkv_score    steps 1-2   window attention (Algorithm 2) and the projected value-row norm (Algorithm 1)
+ *   criticalkv_select   steps 3-4   scores per KV head, budgets, two-stage top-k (Algorithm 1)
+ *   criticalkv_compact  step  5     gather of the retained rows (Algorithm 1, "add K_i, V_i to K_hat, V_hat")
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer unless the argument is documented as host memory.  The caller owns all
+ *     buffers, including the workspace; the library allocates device memory only in criticalkv_create (one status
+ *     word).
+ *   - Calls only enqueue work on the given CUDA stream (a cudaStream_t passed as void*, NULL = legacy default stream)
+ *     and return; they never synchronise, except criticalkv_device_status.
+ *   - Return value: a criticalkv_status.  Argument errors are found on the host before any launch.  A device-side
+ *     anomaly (a bounded wait that ran out) sets the handle's device status word; kernels still terminate.
+ *   - Identical inputs give bit-identical outputs (no order-dependent floating-point atomics).
+ *   - Data pointers must be 16-byte aligned; strides (in elements) must keep every row 16-byte aligned.
+ *   - One handle per host thread / stream.
+ *
+ * Layouts (innermost index contiguous; nb = batch x layers handled by one call)
+ *   Qw  [nb, Hq,  w, dh]   the last w query rows of each query head (the observation window)
+ *   K,V [nb, Hkv, n, dh]   the KV cache; query head h reads KV head h / (Hq/Hkv)
+ *   WO  [nbw, Hq, dh, dm]  head h's rows h*dh .. (h+1)*dh-1 of the (Hq*dh) x dm output projection (Eq. 2: o = A V W^O);
+ *                          nbw = nb, or 1 when CKV_FLAG_WO_SHARED is set
+ *   attn, vnorm [nb, Hq, n] float32
+ *   idx [nb, Btot] int32, offsets [nb, Hkv+1] int32, stage [nb, Btot] uint8 (1 = stage 1, 2 = stage 2)
+ *   K_out, V_out [nb, Btot, dh], same element type as K, V
+ *   Btot = Hkv * budget (uniform), budget (flattened adaptive), or the capacity given by the caller (given budgets).
+ */
+#ifndef CRITICALKV_H_
+#define CRITICALKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define CKV_API __attribute__((visibility("default")))
+#else
+#define CKV_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct criticalkv_handle_s* criticalkv_handle;
+
+typedef enum {
+  CKV_OK = 0,
+  CKV_EINVAL = -1,      /* bad argument (null pointer, shape, budget out of range)            */
+  CKV_ENOTSUP = -2,     /* valid request this build does not implement                        */
+  CKV_EALIGN = -3,      /* pointer or stride not 16-byte aligned                              */
+  CKV_EWORKSPACE = -4,  /* workspace smaller than criticalkv_workspace_bytes reports          */
+  CKV_ECUDA = -5,       /* a CUDA runtime/driver call failed (see criticalkv_last_cuda_error) */
+  CKV_ETIMEOUT = -6     /* a bounded device-side wait ran out (read via criticalkv_device_status) */
+} criticalkv_status;
+
+typedef enum { CKV_F32 = 0, CKV_BF16 = 1 } criticalkv_dtype;
+typedef enum { CKV_BUDGET_UNIFORM = 0, CKV_BUDGET_FLAT_ADAPTIVE = 1, CKV_BUDGET_GIVEN = 2 } criticalkv_budget_mode;
+typedef enum { CKV_NORM_L1 = 0 } criticalkv_norm;
+
+enum {
+  CKV_FLAG_WO_SHARED = 1u << 0,   /* WO has no nb dimension (one projection for the whole call)             */
+  CKV_FLAG_FORCE_SIMT = 1u << 1   /* bf16 only: use the CUDA-core kernels instead of the tensor-core ones   */
+};
+
+/* Problem descriptor (plain data, copied by every call). */
+typedef struct {
+  int32_t nb;            /* >= 1                                                                        */
+  int32_t Hq, Hkv;       /* Hq % Hkv == 0, Hkv <= 64                                                    */
+  int32_t dh;            /* head dim: 64 or 128                                                         */
+  int32_t dm;            /* model dim, multiple of 8                                                    */
+  int32_t n;             /* cached entries per head, >= w                                               */
+  int32_t w;             /* observation window (Algorithm 2: n'), 1..64                                 */
+  int32_t pool_k;        /* max-pool kernel, odd, 1..63 (Algorithm 2: maxpooling; 7 in the paper)       */
+  int32_t dtype;         /* criticalkv_dtype of Qw, K, V, WO, K_out, V_out                              */
+  float scale;           /* logit scale of Eq. 2; <= 0 selects 1/sqrt(dh)                               */
+  float alpha;           /* stage split of Algorithm 1 in [0,1]: b' = floor(alpha*b), b'' = b - b'      */
+  float eps;             /* Algorithm 1: (A + eps) * norm; the paper uses 1e-4                          */
+  int32_t budget_mode;   /* criticalkv_budget_mode                                                      */
+  int32_t norm;          /* criticalkv_norm                                                             */
+  int64_t budget;        /* UNIFORM: B per KV head (<= n); FLAT_ADAPTIVE: B_total per nb slice
+                            (<= Hkv*n); GIVEN: capacity Btot of idx per nb slice (>= sum of budgets)    */
+  uint32_t flags;        /* CKV_FLAG_*                                                                  */
+  uint32_t reserved;     /* must be 0                                                                   */
+  /* Element strides of Qw / K / V for the nb, head and row (token) index; 0 selects the dense default. */
+  int64_t q_stride[3];
+  int64_t k_stride[3];
+  int64_t v_stride[3];
+} criticalkv_desc;
+
+/* Create / destroy a handle bound to CUDA device `device`.  create allocates one device status word. */
+CKV_API int criticalkv_create(criticalkv_handle* out, int device);
+CKV_API int criticalkv_destroy(criticalkv_handle h);
+
+/* Workspace sizes in bytes for score and select (host computation, no CUDA call); compact needs none. */
+CKV_API int criticalkv_workspace_bytes(const criticalkv_desc* d, size_t* score_bytes, size_t* select_bytes);
+
+/*
+ * Steps 1-2.  attn[nb,Hq,n]: per query head the causal softmax of the w window queries over all n keys (window row
+ * j sits at position n-w+j and sees keys i <= n-w+j), averaged over the window and max-pooled along the sequence
+ * (Algorithm 2; Eq. 2).  vnorm[nb,Hq,n]: L1 norm of each value row projected through that head's slice of W^O
+ * (Algorithm 1, "L1 norm of each row of V W^O"; Theorem 3.3).  The n x dm product is never written to memory.
+ * Either output may be NULL to skip that half.  ws: workspace of at least score_bytes, 256-byte aligned.
+ */
+CKV_API int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K,
+                             const void* V, const void* WO, float* attn, float* vnorm, void* ws, size_t ws_bytes,
+                             void* stream);
+
+/*
+ * Steps 3-4.  Per KV head g: a_g = mean over the group's query heads of attn, c_g = mean of (attn + eps) * vnorm
+ * (Algorithm 1), each +, *, / a separately rounded float32 operation, heads summed in increasing order.  Budgets:
+ * uniform, flattened top-B_total of a over (g, i) counted per head (Algorithm 2, budget allocation), or read from
+ * budgets_in[nb,Hkv] (device).  Then stage 1 keeps the b' largest a_g, stage 2 the b'' largest c_g among the rest
+ * (Algorithm 1); ties go to the lower index; idx is ascending inside each head's segment
+ * [offsets[g], offsets[g+1]).  stage may be NULL.  With given budgets whose sum is below the capacity the tail of
+ * idx is left untouched; budgets outside [0, n] or beyond the capacity are clipped and flagged in the status word.
+ */
+CKV_API int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, const float* attn, const float* vnorm,
+                              const int32_t* budgets_in, int32_t* idx, int32_t* offsets, uint8_t* stage, void* ws,
+                              size_t ws_bytes, void* stream);
+
+/* Step 5.  K_out[nb, r, :] = K[nb, g, idx[nb, r], :] for r in head g's segment, same for V (bit copy). */
+CKV_API int criticalkv_compact(criticalkv_handle h, const criticalkv_desc* d, const void* K, const void* V,
+                               const int32_t* idx, const int32_t* offsets, void* K_out, void* V_out, void* stream);
+
+/* The three calls above back to back on one stream.  ws must hold max(score_bytes, select_bytes). */
+CKV_API int criticalkv_compress(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K,
+                                const void* V, const void* WO, const int32_t* budgets_in, float* attn, float* vnorm,
+                                int32_t* idx, int32_t* offsets, uint8_t* stage, void* K_out, void* V_out, void* ws,
+                                size_t ws_bytes, void* stream);
+
+/* Reads the device status word (synchronises `stream` first), clears it, and returns it in *out. */
+CKV_API int criticalkv_device_status(criticalkv_handle h, void* stream, int* out);
+
+CKV_API const char* criticalkv_status_string(int status);
+/* Last CUDA error string seen by this handle ("" if none); valid until the next call on the handle. */
+CKV_API const char* criticalkv_last_cuda_error(criticalkv_handle h);
+/* Which kernels the last criticalkv_score on this handle launched: bit0 tensor-core window attention,
+   bit1 tensor-core projection norm, bit2 CUDA-core window attention, bit3 CUDA-core projection norm. */
+CKV_API int criticalkv_last_path(criticalkv_handle h);
+/* Number of kernel launches this handle has issued since it was created. */
+CKV_API int64_t criticalkv_launch_count(criticalkv_handle h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CRITICALKV_H_ */

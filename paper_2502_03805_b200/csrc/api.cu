@@ -1,0 +1,298 @@
+// C ABI of libcriticalkv: argument validation, workspace carving and kernel dispatch.
+// All checks run on the host before the first launch; nothing here synchronises except criticalkv_device_status.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "ckv_internal.h"
+
+struct criticalkv_handle_s {
+  int device;
+  int sm_count;
+  int cc_major, cc_minor;
+  int* status_word;  // device
+  int last_path;
+  long long launches;
+  char cuda_error[256];
+};
+
+namespace {
+
+using ckv::Dims;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int record_cuda(criticalkv_handle h, cudaError_t e) {
+  if (e == cudaSuccess) return CKV_OK;
+  if (h) snprintf(h->cuda_error, sizeof(h->cuda_error), "%s: %s", cudaGetErrorName(e), cudaGetErrorString(e));
+  return CKV_ECUDA;
+}
+
+// Validates the descriptor and resolves defaults.  Returns CKV_OK or the status to hand back.
+int resolve(const criticalkv_desc* d, Dims* o) {
+  if (!d || !o) return CKV_EINVAL;
+  if (d->nb < 1 || d->Hq < 1 || d->Hkv < 1 || d->Hq % d->Hkv != 0) return CKV_EINVAL;
+  if (d->Hkv > 64) return CKV_ENOTSUP;
+  if (d->dh != 64 && d->dh != 128) return CKV_ENOTSUP;
+  if (d->dm < 8 || d->dm % 8 != 0) return CKV_EINVAL;
+  if (d->w < 1) return CKV_EINVAL;
+  if (d->w > 64) return CKV_ENOTSUP;
+  if (d->n < d->w) return CKV_EINVAL;
+  if (d->pool_k < 1 || d->pool_k % 2 == 0) return CKV_EINVAL;
+  if (d->pool_k > 63) return CKV_ENOTSUP;
+  if (d->dtype != CKV_F32 && d->dtype != CKV_BF16) return CKV_EINVAL;
+  if (!(d->alpha >= 0.f && d->alpha <= 1.f)) return CKV_EINVAL;
+  if (!(d->eps >= 0.f) || !isfinite(d->eps)) return CKV_EINVAL;
+  if (d->norm != CKV_NORM_L1) return CKV_ENOTSUP;
+  if (d->reserved != 0) return CKV_EINVAL;
+  if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT)) return CKV_EINVAL;
+  if (d->budget < 0) return CKV_EINVAL;
+  if ((long long)d->n * d->Hkv > 0x7fffffffLL) return CKV_ENOTSUP;
+  o->nb = d->nb; o->Hq = d->Hq; o->Hkv = d->Hkv; o->G = d->Hq / d->Hkv;
+  o->dh = d->dh; o->dm = d->dm; o->n = d->n; o->w = d->w; o->kp = d->pool_k; o->dtype = d->dtype;
+  o->scale = d->scale > 0.f ? d->scale : (float)(1.0 / sqrt((double)d->dh));
+  o->alpha = d->alpha; o->eps = d->eps;
+  o->budget_mode = d->budget_mode; o->budget = d->budget;
+  switch (d->budget_mode) {
+    case CKV_BUDGET_UNIFORM:
+      if (d->budget > d->n) return CKV_EINVAL;
+      o->btot = (long long)d->budget * d->Hkv;
+      break;
+    case CKV_BUDGET_FLAT_ADAPTIVE:
+    case CKV_BUDGET_GIVEN:
+      if (d->budget > (long long)d->n * d->Hkv) return CKV_EINVAL;
+      o->btot = d->budget;
+      break;
+    default:
+      return CKV_EINVAL;
+  }
+  if (o->btot > 0x7fffffffLL) return CKV_ENOTSUP;
+  o->wo_shared = (d->flags & CKV_FLAG_WO_SHARED) ? 1 : 0;
+  const long long dq[3] = {(long long)d->Hq * d->w * d->dh, (long long)d->w * d->dh, d->dh};
+  const long long dk[3] = {(long long)d->Hkv * d->n * d->dh, (long long)d->n * d->dh, d->dh};
+  const int vec = d->dtype == CKV_F32 ? 4 : 8;  // elements per 16 bytes
+  for (int i = 0; i < 3; ++i) {
+    o->qs[i] = d->q_stride[i] ? d->q_stride[i] : dq[i];
+    o->ks[i] = d->k_stride[i] ? d->k_stride[i] : dk[i];
+    o->vs[i] = d->v_stride[i] ? d->v_stride[i] : dk[i];
+    if (o->qs[i] < 0 || o->ks[i] < 0 || o->vs[i] < 0) return CKV_EINVAL;
+    if (o->qs[i] % vec || o->ks[i] % vec || o->vs[i] % vec) return CKV_EALIGN;
+  }
+  if (o->qs[2] < d->dh || o->ks[2] < d->dh || o->vs[2] < d->dh) return CKV_EINVAL;
+  return CKV_OK;
+}
+
+struct ScoreLayout {
+  size_t part_m, part_l, rowstat, abar, total;
+};
+ScoreLayout score_layout(const Dims& d) {
+  ScoreLayout L;
+  const size_t rows = (size_t)d.nb * d.Hq * d.w;
+  const size_t nchunks = (d.n + ckv::kAttnChunk - 1) / ckv::kAttnChunk;
+  size_t off = 0;
+  L.part_m = off; off = align_up(off + rows * nchunks * sizeof(float), 256);
+  L.part_l = off; off = align_up(off + rows * nchunks * sizeof(float), 256);
+  L.rowstat = off; off = align_up(off + rows * 2 * sizeof(float), 256);
+  L.abar = off; off = align_up(off + (size_t)d.nb * d.Hq * d.n * sizeof(float), 256);
+  L.total = off;
+  return L;
+}
+struct SelectLayout {
+  size_t a, c, budgets, total;
+};
+SelectLayout select_layout(const Dims& d) {
+  SelectLayout L;
+  const size_t per = (size_t)d.nb * d.Hkv * d.n * sizeof(float);
+  size_t off = 0;
+  L.a = off; off = align_up(off + per, 256);
+  L.c = off; off = align_up(off + per, 256);
+  L.budgets = off; off = align_up(off + (size_t)d.nb * d.Hkv * sizeof(int32_t), 256);
+  L.total = off;
+  return L;
+}
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; prev = -1; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    if (prev == dev) prev = -1;
+  }
+  ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace
+
+extern "C" {
+
+int criticalkv_create(criticalkv_handle* out, int device) {
+  if (!out) return CKV_EINVAL;
+  *out = nullptr;
+  int count = 0;
+  cudaError_t e = cudaGetDeviceCount(&count);
+  if (e != cudaSuccess) return CKV_ECUDA;
+  if (device < 0 || device >= count) return CKV_EINVAL;
+  criticalkv_handle h = new (std::nothrow) criticalkv_handle_s();
+  if (!h) return CKV_EINVAL;
+  memset(h, 0, sizeof(*h));
+  h->device = device;
+  DeviceGuard guard(device);
+  cudaDeviceProp prop;
+  if (!guard.ok || (e = cudaGetDeviceProperties(&prop, device)) != cudaSuccess ||
+      (e = cudaMalloc(&h->status_word, sizeof(int))) != cudaSuccess ||
+      (e = cudaMemset(h->status_word, 0, sizeof(int))) != cudaSuccess) {
+    delete h;
+    return CKV_ECUDA;
+  }
+  h->sm_count = prop.multiProcessorCount;
+  h->cc_major = prop.major;
+  h->cc_minor = prop.minor;
+  *out = h;
+  return CKV_OK;
+}
+
+int criticalkv_destroy(criticalkv_handle h) {
+  if (!h) return CKV_EINVAL;
+  DeviceGuard guard(h->device);
+  if (h->status_word) cudaFree(h->status_word);
+  delete h;
+  return CKV_OK;
+}
+
+int criticalkv_workspace_bytes(const criticalkv_desc* d, size_t* score_bytes, size_t* select_bytes) {
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (score_bytes) *score_bytes = score_layout(dd).total;
+  if (select_bytes) *select_bytes = select_layout(dd).total;
+  return CKV_OK;
+}
+
+int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K, const void* V,
+                     const void* WO, float* attn, float* vnorm, void* ws, size_t ws_bytes, void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (!attn && !vnorm) return CKV_EINVAL;
+  if (attn && (!Qw || !K)) return CKV_EINVAL;
+  if (vnorm && (!V || !WO)) return CKV_EINVAL;
+  if (!ws) return CKV_EINVAL;
+  if (!aligned16(Qw) || !aligned16(K) || !aligned16(V) || !aligned16(WO) || !aligned16(attn) || !aligned16(vnorm) ||
+      (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return CKV_EALIGN;
+  const ScoreLayout L = score_layout(dd);
+  if (ws_bytes < L.total) return CKV_EWORKSPACE;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* base = (char*)ws;
+  ckv::ScoreWorkspace sw{(float*)(base + L.part_m), (float*)(base + L.part_l), (float*)(base + L.rowstat),
+                         (float*)(base + L.abar)};
+  int launches = 0, path = 0;
+  cudaError_t e = cudaSuccess;
+  if (attn) {
+    e = ckv::launch_window_attn_simt(dd, Qw, K, attn, sw, st, &launches);
+    path |= 4;
+  }
+  if (e == cudaSuccess && vnorm) {
+    e = ckv::launch_vnorm_simt(dd, V, WO, vnorm, st, &launches);
+    path |= 8;
+  }
+  h->launches += launches;
+  h->last_path = path;
+  return record_cuda(h, e);
+}
+
+int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, const float* attn, const float* vnorm,
+                      const int32_t* budgets_in, int32_t* idx, int32_t* offsets, uint8_t* stage, void* ws,
+                      size_t ws_bytes, void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (!attn || !vnorm || !idx || !offsets || !ws) return CKV_EINVAL;
+  if (dd.budget_mode == CKV_BUDGET_GIVEN && !budgets_in) return CKV_EINVAL;
+  if (!aligned16(attn) || !aligned16(vnorm) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
+      (reinterpret_cast<uintptr_t>(offsets) & 3u) || (reinterpret_cast<uintptr_t>(budgets_in) & 3u) ||
+      (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return CKV_EALIGN;
+  const SelectLayout L = select_layout(dd);
+  if (ws_bytes < L.total) return CKV_EWORKSPACE;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  char* base = (char*)ws;
+  ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets)};
+  int launches = 0;
+  cudaError_t e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, (cudaStream_t)stream,
+                                     &launches, h->status_word);
+  h->launches += launches;
+  return record_cuda(h, e);
+}
+
+int criticalkv_compact(criticalkv_handle h, const criticalkv_desc* d, const void* K, const void* V,
+                       const int32_t* idx, const int32_t* offsets, void* K_out, void* V_out, void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (!K || !V || !idx || !offsets || !K_out || !V_out) return CKV_EINVAL;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(K_out) || !aligned16(V_out) ||
+      (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(offsets) & 3u))
+    return CKV_EALIGN;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  if (dd.btot == 0) return CKV_OK;
+  int launches = 0;
+  cudaError_t e = ckv::launch_compact(dd, K, V, idx, offsets, K_out, V_out, (cudaStream_t)stream, &launches);
+  h->launches += launches;
+  return record_cuda(h, e);
+}
+
+int criticalkv_compress(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K, const void* V,
+                        const void* WO, const int32_t* budgets_in, float* attn, float* vnorm, int32_t* idx,
+                        int32_t* offsets, uint8_t* stage, void* K_out, void* V_out, void* ws, size_t ws_bytes,
+                        void* stream) {
+  if (!attn || !vnorm) return CKV_EINVAL;
+  int rc = criticalkv_score(h, d, Qw, K, V, WO, attn, vnorm, ws, ws_bytes, stream);
+  if (rc != CKV_OK) return rc;
+  rc = criticalkv_select(h, d, attn, vnorm, budgets_in, idx, offsets, stage, ws, ws_bytes, stream);
+  if (rc != CKV_OK) return rc;
+  return criticalkv_compact(h, d, K, V, idx, offsets, K_out, V_out, stream);
+}
+
+int criticalkv_device_status(criticalkv_handle h, void* stream, int* out) {
+  if (!h || !out) return CKV_EINVAL;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  int v = 0;
+  cudaError_t e = cudaMemcpyAsync(&v, h->status_word, sizeof(int), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaMemsetAsync(h->status_word, 0, sizeof(int), st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  *out = v;
+  return record_cuda(h, e);
+}
+
+const char* criticalkv_status_string(int s) {
+  switch (s) {
+    case CKV_OK: return "ok";
+    case CKV_EINVAL: return "invalid argument";
+    case CKV_ENOTSUP: return "not supported";
+    case CKV_EALIGN: return "pointer or stride not 16-byte aligned";
+    case CKV_EWORKSPACE: return "workspace too small";
+    case CKV_ECUDA: return "CUDA call failed";
+    case CKV_ETIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+const char* criticalkv_last_cuda_error(criticalkv_handle h) { return h ? h->cuda_error : ""; }
+int criticalkv_last_path(criticalkv_handle h) { return h ? h->last_path : 0; }
+int64_t criticalkv_launch_count(criticalkv_handle h) { return h ? h->launches : 0; }
+
+}  // extern "C"

@@ -1,0 +1,49 @@
+// Internal declarations shared by the translation units of libcriticalkv (not part of the public ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "criticalkv.h"
+
+namespace ckv {
+
+// Resolved problem description handed to the launchers (host side).
+struct Dims {
+  int nb, Hq, Hkv, G, dh, dm, n, w, kp;
+  int dtype;
+  float scale, alpha, eps;
+  int budget_mode;
+  long long budget;   // as in criticalkv_desc
+  long long btot;     // capacity of idx per nb slice
+  int wo_shared;
+  long long qs[3], ks[3], vs[3];  // element strides: nb, head, row
+};
+
+// Keys of the window-attention kernels are processed in chunks of this many tokens (one CTA each).
+constexpr int kAttnChunk = 256;
+
+struct ScoreWorkspace {   // carved out of the caller's workspace by the API layer
+  float* part_m;    // [nb*Hq*w, nchunks]   partial row maxima
+  float* part_l;    // [nb*Hq*w, nchunks]   partial row sums of exp
+  float* rowstat;   // [nb*Hq*w, 2]         final (max, 1/(w*sum))
+  float* abar;      // [nb*Hq, n]           window-mean attention before pooling
+};
+
+struct SelectWorkspace {
+  float* a;         // [nb, Hkv, n]
+  float* c;         // [nb, Hkv, n]
+  int32_t* budgets; // [nb, Hkv]
+};
+
+// ---- launchers (each returns the first CUDA error of its launches) ----
+cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K, float* attn,
+                                    const ScoreWorkspace& ws, cudaStream_t st, int* launches);
+cudaError_t launch_vnorm_simt(const Dims& d, const void* V, const void* WO, float* vnorm, cudaStream_t st,
+                              int* launches);
+cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
+                          int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
+                          cudaStream_t st, int* launches, int* status_word);
+cudaError_t launch_compact(const Dims& d, const void* K, const void* V, const int32_t* idx, const int32_t* offsets,
+                           void* K_out, void* V_out, cudaStream_t st, int* launches);
+
+}  // namespace ckv

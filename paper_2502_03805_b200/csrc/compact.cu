@@ -1,0 +1,70 @@
+// Step 5: compaction of the retained entries (Algorithm 1: "add K_i, V_i to K_hat, V_hat").
+// K_out[nb, r, :] = K[nb, g, idx[nb, r], :] for every r in head g's segment [offsets[g], offsets[g+1]); same for V.
+// Pure data movement: every row is copied as 16-byte vectors, one lane per vector, consecutive lanes on consecutive
+// vectors of a row (a 256-byte bf16 row of head_dim 128 is 16 lanes), rows of one head read in ascending order.
+#include "ckv_internal.h"
+
+namespace ckv {
+namespace {
+
+struct CompactArgs {
+  const char* K;
+  const char* V;
+  const int32_t* idx;
+  const int32_t* offsets;
+  char* K_out;
+  char* V_out;
+  int Hkv, n;
+  int vec_per_row;          // 16-byte vectors per row
+  long long btot;
+  long long ks[3], vs[3];   // byte strides: nb, head, row
+};
+
+constexpr int kThreads = 256;
+
+__global__ void __launch_bounds__(kThreads) compact_kernel(CompactArgs p) {
+  __shared__ int32_t offs[65];
+  const int b = blockIdx.y;
+  for (int q = threadIdx.x; q <= p.Hkv; q += kThreads) offs[q] = p.offsets[(long long)b * (p.Hkv + 1) + q];
+  __syncthreads();
+  const long long total = min((long long)offs[p.Hkv], p.btot);
+  const int rows_per_cta = kThreads / p.vec_per_row;
+  const int lane = threadIdx.x % p.vec_per_row, sub = threadIdx.x / p.vec_per_row;
+  if (sub >= rows_per_cta) return;
+  for (long long r = (long long)blockIdx.x * rows_per_cta + sub; r < total; r += (long long)gridDim.x * rows_per_cta) {
+    int g = 0;
+    while (g + 1 < p.Hkv && r >= offs[g + 1]) ++g;
+    const int src = p.idx[(long long)b * p.btot + r];
+    if (src < 0 || src >= p.n) continue;
+    const long long ko = b * p.ks[0] + g * p.ks[1] + (long long)src * p.ks[2] + lane * 16LL;
+    const long long vo = b * p.vs[0] + g * p.vs[1] + (long long)src * p.vs[2] + lane * 16LL;
+    const long long oo = ((long long)b * p.btot + r) * p.vec_per_row * 16LL + lane * 16LL;
+    const uint4 kv = *reinterpret_cast<const uint4*>(p.K + ko);
+    const uint4 vv = *reinterpret_cast<const uint4*>(p.V + vo);
+    *reinterpret_cast<uint4*>(p.K_out + oo) = kv;
+    *reinterpret_cast<uint4*>(p.V_out + oo) = vv;
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_compact(const Dims& d, const void* K, const void* V, const int32_t* idx, const int32_t* offsets,
+                           void* K_out, void* V_out, cudaStream_t st, int* launches) {
+  const int es = d.dtype == CKV_F32 ? 4 : 2;
+  CompactArgs p;
+  p.K = (const char*)K; p.V = (const char*)V; p.idx = idx; p.offsets = offsets;
+  p.K_out = (char*)K_out; p.V_out = (char*)V_out;
+  p.Hkv = d.Hkv; p.n = d.n; p.btot = d.btot;
+  p.vec_per_row = d.dh * es / 16;
+  for (int i = 0; i < 3; ++i) { p.ks[i] = d.ks[i] * es; p.vs[i] = d.vs[i] * es; }
+  const int rows_per_cta = kThreads / p.vec_per_row;
+  long long ctas = (d.btot + rows_per_cta - 1) / rows_per_cta;
+  if (ctas < 1) ctas = 1;
+  if (ctas > 148 * 16) ctas = 148 * 16;
+  dim3 grid((unsigned)ctas, d.nb);
+  compact_kernel<<<grid, kThreads, 0, st>>>(p);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace ckv

@@ -1,0 +1,299 @@
+// Steps 3-4: scores per KV head, budgets, and the two-stage top-k of Algorithm 1.
+//
+//   group_reduce : a_g = mean_h attn_h, c_g = mean_h (attn_h + eps) * vnorm_h over the query heads of a KV group,
+//                  every operation a separately rounded float32 op in a fixed order (the selection is decided in
+//                  exactly this arithmetic)
+//   adaptive     : flattened top-B_total of a over (g, i), counted per head (Algorithm 2, budget allocation)
+//   two_stage    : per (nb, KV head): stage 1 = b' largest a_g, stage 2 = b'' largest c_g among the rest,
+//                  b' = floor(alpha * b); ties go to the lower index; indices written in ascending order
+//
+// Top-k is a radix *select* (4 passes of 8 bits over order-preserving integer keys) followed by an ordered walk that
+// resolves ties by index and compacts with warp ballots: no sort, no floating-point atomics, bit-reproducible.
+#include "ckv_internal.h"
+
+namespace ckv {
+namespace {
+
+constexpr int kSelThreads = 1024;
+constexpr int kSelWarps = kSelThreads / 32;
+
+__device__ __forceinline__ uint32_t order_key(float x) {
+  const uint32_t u = __float_as_uint(x);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void group_reduce_kernel(const float* __restrict__ attn, const float* __restrict__ vnorm,
+                                    float* __restrict__ a, float* __restrict__ c, int Hq, int Hkv, int G, int n,
+                                    float eps) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int g = blockIdx.y, b = blockIdx.z;
+  const long long h0 = (long long)b * Hq + (long long)g * G;
+  float p = attn[h0 * n + i];
+  float sa = p;
+  float sc = __fmul_rn(__fadd_rn(p, eps), vnorm[h0 * n + i]);
+  for (int q = 1; q < G; ++q) {
+    p = attn[(h0 + q) * n + i];
+    sa = __fadd_rn(sa, p);
+    sc = __fadd_rn(sc, __fmul_rn(__fadd_rn(p, eps), vnorm[(h0 + q) * n + i]));
+  }
+  const float Gf = (float)G;
+  float av = __fdiv_rn(sa, Gf), cv = __fdiv_rn(sc, Gf);
+  if (av == 0.f) av = 0.f;  // -0 and +0 must order alike
+  if (cv == 0.f) cv = 0.f;
+  const long long o = ((long long)b * Hkv + g) * n + i;
+  a[o] = av;
+  c[o] = cv;
+}
+
+struct SelectShared {
+  uint32_t hist[kSelWarps][256];
+  uint32_t total[256];
+  uint32_t warp_cnt[kSelWarps];
+  uint32_t prefix;
+  uint32_t krem;
+};
+
+__device__ __forceinline__ bool excluded(const uint32_t* excl, long long i) {
+  return excl != nullptr && ((excl[i >> 5] >> (i & 31)) & 1u);
+}
+
+// Finds the k-th largest key among the candidates (all i in [0, count) not excluded), 1 <= k <= #candidates.
+// On return (all threads): *T = that key, *r = how many entries equal to T belong to the top k.
+__device__ void radix_select(const float* __restrict__ keys, long long count, const uint32_t* excl, uint32_t k,
+                             SelectShared& sh, uint32_t* T, uint32_t* r) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { sh.prefix = 0; sh.krem = k; }
+  uint32_t known = 0;  // mask of the key bits fixed so far
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int e = tid; e < kSelWarps * 256; e += kSelThreads) (&sh.hist[0][0])[e] = 0;
+    __syncthreads();
+    const uint32_t prefix = sh.prefix;
+    for (long long i = tid; i < count; i += kSelThreads) {
+      if (excluded(excl, i)) continue;
+      const uint32_t key = order_key(keys[i]);
+      if ((key & known) == prefix) atomicAdd(&sh.hist[warp][(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 256) {
+      uint32_t s = 0;
+      for (int wq = 0; wq < kSelWarps; ++wq) s += sh.hist[wq][tid];
+      sh.total[tid] = s;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // lane l owns digits 8l .. 8l+7; find the digit at which the count from the top reaches krem
+      uint32_t mine = 0;
+      for (int q = 0; q < 8; ++q) mine += sh.total[lane * 8 + q];
+      uint32_t above = mine;  // inclusive suffix sum over lanes >= lane
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, above, o);
+        if (lane + o < 32) above += v;
+      }
+      above -= mine;  // keys in strictly higher lanes
+      const uint32_t krem = sh.krem;
+      if (above < krem && krem <= above + mine) {
+        uint32_t acc = above;
+        for (int q = 7; q >= 0; --q) {
+          const uint32_t cnt = sh.total[lane * 8 + q];
+          if (acc + cnt >= krem) {
+            sh.prefix = prefix | ((uint32_t)(lane * 8 + q) << shift);
+            sh.krem = krem - acc;
+            break;
+          }
+          acc += cnt;
+        }
+      }
+    }
+    known |= 0xffu << shift;
+    __syncthreads();
+  }
+  *T = sh.prefix;
+  *r = sh.krem;
+  __syncthreads();
+}
+
+// Ordered walk over [0, n): sets bit i of out[] iff key_i > T, or key_i == T and fewer than r equal candidates
+// precede i.  Warp q owns the contiguous word range [q * wpw, (q + 1) * wpw).
+__device__ void mark_selected(const float* __restrict__ keys, int n, const uint32_t* excl, uint32_t T, uint32_t r,
+                              bool any, uint32_t* out, SelectShared& sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nwords = (n + 31) / 32;
+  const int wpw = (nwords + kSelWarps - 1) / kSelWarps;
+  const int w0 = min(warp * wpw, nwords), w1 = min(w0 + wpw, nwords);
+  uint32_t eq_count = 0;
+  for (int q = w0; q < w1; ++q) {
+    const int i = q * 32 + lane;
+    const bool valid = any && i < n && !excluded(excl, i);
+    const bool eq = valid && order_key(keys[i]) == T;
+    eq_count += __popc(__ballot_sync(0xffffffffu, eq));
+  }
+  if (lane == 0) sh.warp_cnt[warp] = eq_count;
+  __syncthreads();
+  uint32_t running = 0;
+  for (int q = 0; q < warp; ++q) running += sh.warp_cnt[q];
+  for (int q = w0; q < w1; ++q) {
+    const int i = q * 32 + lane;
+    const bool valid = any && i < n && !excluded(excl, i);
+    const uint32_t key = valid ? order_key(keys[i]) : 0u;
+    const bool eq = valid && key == T;
+    const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
+    const bool take = eq && (running + __popc(eqm & ((1u << lane) - 1u)) < r);
+    const uint32_t word = __ballot_sync(0xffffffffu, (valid && key > T) || take);
+    if (lane == 0) out[q] = word;
+    running += __popc(eqm);
+  }
+  __syncthreads();
+}
+
+struct TwoStageArgs {
+  const float* a;
+  const float* c;
+  const int32_t* budgets;  // [nb, Hkv] or nullptr for uniform
+  int32_t* idx;
+  int32_t* offsets;
+  uint8_t* stage;
+  int* status;
+  int Hkv, n;
+  long long uniform_b, btot;
+  float alpha;
+};
+
+__global__ void __launch_bounds__(kSelThreads) two_stage_kernel(TwoStageArgs p) {
+  extern __shared__ __align__(16) uint32_t dyn[];
+  __shared__ SelectShared sh;
+  const int g = blockIdx.x, b = blockIdx.y;
+  const int n = p.n;
+  const int nwords = (n + 31) / 32;
+  uint32_t* sel1 = dyn;
+  uint32_t* sel2 = dyn + nwords;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+  // this head's budget and the start of its segment
+  long long off = 0, bud;
+  bool clipped = false;
+  if (p.budgets == nullptr) {
+    bud = p.uniform_b;
+    off = (long long)g * bud;
+  } else {
+    const int32_t* bb = p.budgets + (long long)b * p.Hkv;
+    for (int q = 0; q < g; ++q) off += min(max((long long)bb[q], 0LL), (long long)n);
+    bud = bb[g];
+    if (bud < 0 || bud > n) { bud = min(max(bud, 0LL), (long long)n); clipped = true; }
+    if (off > p.btot) { off = p.btot; clipped = true; }
+    if (off + bud > p.btot) { bud = p.btot - off; clipped = true; }
+  }
+  if (clipped && threadIdx.x == 0) atomicExch(p.status, (int)CKV_EINVAL);
+  long long b1 = (long long)floor((double)p.alpha * (double)bud);
+  b1 = min(max(b1, 0LL), bud);
+  const long long b2 = bud - b1;
+
+  const float* ag = p.a + ((long long)b * p.Hkv + g) * n;
+  const float* cg = p.c + ((long long)b * p.Hkv + g) * n;
+
+  uint32_t T = 0, r = 0;
+  if (b1 > 0) radix_select(ag, n, nullptr, (uint32_t)b1, sh, &T, &r);
+  mark_selected(ag, n, nullptr, T, r, b1 > 0, sel1, sh);
+  if (b2 > 0) radix_select(cg, n, sel1, (uint32_t)b2, sh, &T, &r);
+  mark_selected(cg, n, sel1, T, r, b2 > 0, sel2, sh);
+
+  // ordered compaction of sel1 | sel2
+  const int wpw = (nwords + kSelWarps - 1) / kSelWarps;
+  const int w0 = min(warp * wpw, nwords), w1 = min(w0 + wpw, nwords);
+  uint32_t cnt = 0;
+  for (int q = w0 + lane; q < w1; q += 32) cnt += __popc(sel1[q] | sel2[q]);
+  for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+  if (lane == 0) sh.warp_cnt[warp] = cnt;
+  __syncthreads();
+  uint32_t running = 0;
+  for (int q = 0; q < warp; ++q) running += sh.warp_cnt[q];
+  int32_t* idx = p.idx + (long long)b * p.btot + off;
+  uint8_t* stage = p.stage ? p.stage + (long long)b * p.btot + off : nullptr;
+  for (int q = w0; q < w1; ++q) {
+    const uint32_t s1 = sel1[q], word = s1 | sel2[q];
+    if ((word >> lane) & 1u) {
+      const uint32_t pos = running + __popc(word & ((1u << lane) - 1u));
+      idx[pos] = q * 32 + lane;
+      if (stage) stage[pos] = ((s1 >> lane) & 1u) ? 1 : 2;
+    }
+    running += __popc(word);
+  }
+  if (threadIdx.x == 0) {
+    p.offsets[(long long)b * (p.Hkv + 1) + g] = (int32_t)off;
+    if (g == p.Hkv - 1) p.offsets[(long long)b * (p.Hkv + 1) + p.Hkv] = (int32_t)(off + bud);
+  }
+}
+
+// Flattened top-B_total over a[nb, Hkv*n]: budgets[g] = #{i : key > T} + the first ties in (g, i) order.
+__global__ void __launch_bounds__(kSelThreads) adaptive_budget_kernel(const float* __restrict__ a,
+                                                                      int32_t* __restrict__ budgets, int Hkv, int n,
+                                                                      long long btotal) {
+  __shared__ SelectShared sh;
+  __shared__ uint32_t cnt_gt[64], cnt_eq[64];
+  const int b = blockIdx.x;
+  const float* ab = a + (long long)b * Hkv * n;
+  int32_t* out = budgets + (long long)b * Hkv;
+  if (btotal <= 0) {
+    if (threadIdx.x < Hkv) out[threadIdx.x] = 0;
+    return;
+  }
+  uint32_t T, r;
+  radix_select(ab, (long long)Hkv * n, nullptr, (uint32_t)btotal, sh, &T, &r);
+  if (threadIdx.x < 64) { cnt_gt[threadIdx.x] = 0; cnt_eq[threadIdx.x] = 0; }
+  __syncthreads();
+  for (int g = 0; g < Hkv; ++g) {
+    uint32_t gt = 0, eq = 0;
+    for (int i = threadIdx.x; i < n; i += kSelThreads) {
+      const uint32_t key = order_key(ab[(long long)g * n + i]);
+      gt += key > T;
+      eq += key == T;
+    }
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    eq = __reduce_add_sync(0xffffffffu, eq);
+    if ((threadIdx.x & 31) == 0) {
+      if (gt) atomicAdd(&cnt_gt[g], gt);
+      if (eq) atomicAdd(&cnt_eq[g], eq);
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t rem = r;
+    for (int g = 0; g < Hkv; ++g) {
+      const uint32_t take = min(cnt_eq[g], rem);
+      out[g] = (int32_t)(cnt_gt[g] + take);
+      rem -= take;
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
+                          int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
+                          cudaStream_t st, int* launches, int* status_word) {
+  dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
+  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, ws.a, ws.c, d.Hq, d.Hkv, d.G, d.n, d.eps);
+  *launches += 1;
+  const int32_t* budgets = nullptr;
+  if (d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
+    adaptive_budget_kernel<<<d.nb, kSelThreads, 0, st>>>(ws.a, ws.budgets, d.Hkv, d.n, d.budget);
+    *launches += 1;
+    budgets = ws.budgets;
+  } else if (d.budget_mode == CKV_BUDGET_GIVEN) {
+    budgets = budgets_in;
+  }
+  TwoStageArgs p;
+  p.a = ws.a; p.c = ws.c; p.budgets = budgets; p.idx = idx; p.offsets = offsets; p.stage = stage;
+  p.status = status_word;
+  p.Hkv = d.Hkv; p.n = d.n; p.uniform_b = d.budget; p.btot = d.btot; p.alpha = d.alpha;
+  const size_t dyn = (size_t)2 * ((d.n + 31) / 32) * sizeof(uint32_t);
+  cudaError_t e = cudaFuncSetAttribute(two_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+  if (e != cudaSuccess) return e;
+  dim3 tgrid(d.Hkv, d.nb);
+  two_stage_kernel<<<tgrid, kSelThreads, dyn, st>>>(p);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+}  // namespace ckv

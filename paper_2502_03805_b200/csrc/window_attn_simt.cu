@@ -1,0 +1,247 @@
+// Step 1 on CUDA cores: observation-window attention (Algorithm 2: softmax of the last w queries over all keys,
+// mean over the window, max-pool along the sequence; softmax and scale as in Eq. 2).
+//
+// Used for float32 inputs and as the bf16 fallback.  Four launches:
+//   partial : one CTA per (256-key chunk, query head, nb): logits of the w window rows against the chunk's keys,
+//             per-row maximum and sum of exponentials of the chunk
+//   combine : per (query head, nb): merges the chunk partials into each row's (max, 1 / (w * sum))
+//   prob    : recomputes the same logits, normalises, sums the w rows -> window-mean attention
+//   pool    : stride-1 centred max-pool with clipped borders
+// A thread owns one key; the w logits of that key live in registers.  The two logit computations run the same
+// instruction sequence, so a logit never exceeds the maximum found for its row.
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "ckv_internal.h"
+
+namespace ckv {
+namespace {
+
+constexpr int kThreads = kAttnChunk;  // one key per thread
+
+template <typename T>
+struct Vec16;  // 16-byte global load, widened to float
+template <>
+struct Vec16<float> {
+  static constexpr int kElems = 4;
+  __device__ static void load(const float* p, float* out) {
+    float4 v = *reinterpret_cast<const float4*>(p);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+  }
+};
+template <>
+struct Vec16<__nv_bfloat16> {
+  static constexpr int kElems = 8;
+  __device__ static void load(const __nv_bfloat16* p, float* out) {
+    uint4 v = *reinterpret_cast<const uint4*>(p);
+    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      out[2 * i] = __uint_as_float(u[i] << 16);
+      out[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
+    }
+  }
+};
+
+__device__ __forceinline__ float to_float(float x) { return x; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+struct AttnArgs {
+  const void* Qw;
+  const void* K;
+  float* part_m;
+  float* part_l;
+  float* rowstat;
+  float* abar;
+  int Hq, G, n, w, nchunks;
+  float scale;
+  long long qs[3], ks[3];
+};
+
+// Logits of window rows 0..WT-1 for this thread's key; rows >= w come out as 0 (their queries are zero-filled).
+template <typename T, int DH, int WT>
+__device__ __forceinline__ void key_logits(const T* krow, const float* q_s, float (&acc)[WT]) {
+#pragma unroll
+  for (int j = 0; j < WT; ++j) acc[j] = 0.f;
+  constexpr int E = Vec16<T>::kElems;
+#pragma unroll 1
+  for (int t = 0; t < DH; t += E) {
+    float kf[E];
+    Vec16<T>::load(krow + t, kf);
+#pragma unroll
+    for (int j = 0; j < WT; ++j) {
+      const float4* qv = reinterpret_cast<const float4*>(q_s + j * DH + t);
+#pragma unroll
+      for (int e4 = 0; e4 < E / 4; ++e4) {
+        float4 q = qv[e4];
+        acc[j] = fmaf(q.x, kf[4 * e4 + 0], acc[j]);
+        acc[j] = fmaf(q.y, kf[4 * e4 + 1], acc[j]);
+        acc[j] = fmaf(q.z, kf[4 * e4 + 2], acc[j]);
+        acc[j] = fmaf(q.w, kf[4 * e4 + 3], acc[j]);
+      }
+    }
+  }
+}
+
+template <typename T, int DH, int WT>
+__device__ __forceinline__ void stage_queries(const AttnArgs& a, int b, int h, float* q_s) {
+  const T* q = reinterpret_cast<const T*>(a.Qw) + b * a.qs[0] + h * a.qs[1];
+  for (int e = threadIdx.x; e < WT * DH; e += kThreads) {
+    int j = e / DH, t = e % DH;
+    q_s[e] = (j < a.w) ? to_float(q[j * a.qs[2] + t]) : 0.f;
+  }
+}
+
+template <typename T, int DH, int WT, bool kProb>
+__global__ void __launch_bounds__(kThreads) attn_pass_kernel(AttnArgs a) {
+  extern __shared__ __align__(16) float smem[];
+  float* q_s = smem;                         // [WT][DH]
+  float* red = smem + WT * DH;               // [8 warps][WT]
+  float* stat = red + (kThreads / 32) * WT;  // [WT][2]
+  const int chunk = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int g = h / a.G;
+  const int i = chunk * kAttnChunk + threadIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+  stage_queries<T, DH, WT>(a, b, h, q_s);
+  const long long row = (long long)(b * a.Hq + h) * a.w;
+  if constexpr (kProb) {
+    for (int e = threadIdx.x; e < 2 * a.w; e += kThreads) stat[e] = a.rowstat[row * 2 + e];
+  }
+  __syncthreads();
+
+  float acc[WT];
+  const bool in_range = i < a.n;
+  if (in_range) {
+    const T* krow = reinterpret_cast<const T*>(a.K) + b * a.ks[0] + g * a.ks[1] + (long long)i * a.ks[2];
+    key_logits<T, DH, WT>(krow, q_s, acc);
+  } else {
+#pragma unroll
+    for (int j = 0; j < WT; ++j) acc[j] = 0.f;
+  }
+  const int first_pos = a.n - a.w;  // sequence position of window row 0
+#pragma unroll
+  for (int j = 0; j < WT; ++j) {
+    const bool visible = in_range && j < a.w && i <= first_pos + j;
+    acc[j] = visible ? acc[j] * a.scale : -INFINITY;
+  }
+
+  if constexpr (kProb) {
+    // normalise with the final row statistics and sum the window rows in increasing row order
+    float s = 0.f;
+#pragma unroll
+    for (int j = 0; j < WT; ++j) {
+      if (j < a.w) {
+        float p = (acc[j] == -INFINITY) ? 0.f : expf(acc[j] - stat[2 * j]) * stat[2 * j + 1];
+        s += p;
+      }
+    }
+    if (in_range) a.abar[(long long)(b * a.Hq + h) * a.n + i] = s;
+  } else {
+    // chunk maximum per row
+#pragma unroll
+    for (int j = 0; j < WT; ++j) {
+      float m = acc[j];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+      if (lane == 0) red[warp * WT + j] = m;
+    }
+    __syncthreads();
+    if (threadIdx.x < WT) {
+      float m = red[threadIdx.x];
+      for (int wq = 1; wq < kThreads / 32; ++wq) m = fmaxf(m, red[wq * WT + threadIdx.x]);
+      stat[threadIdx.x] = m;
+    }
+    __syncthreads();
+    // chunk sum of exp(logit - chunk max)
+#pragma unroll
+    for (int j = 0; j < WT; ++j) {
+      float e = (acc[j] == -INFINITY) ? 0.f : expf(acc[j] - stat[j]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+      if (lane == 0) red[warp * WT + j] = e;
+    }
+    __syncthreads();
+    if (threadIdx.x < a.w) {
+      float l = red[threadIdx.x];
+      for (int wq = 1; wq < kThreads / 32; ++wq) l += red[wq * WT + threadIdx.x];
+      const long long o = (row + threadIdx.x) * a.nchunks + chunk;
+      a.part_m[o] = stat[threadIdx.x];
+      a.part_l[o] = l;
+    }
+  }
+}
+
+// Merge chunk partials: M = max_c m_c, L = sum_c l_c * exp(m_c - M); store (M, 1 / (w * L)).
+__global__ void attn_combine_kernel(const float* part_m, const float* part_l, float* rowstat, int rows, int nchunks,
+                                    int w) {
+  const int r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= rows) return;
+  const float* pm = part_m + (long long)r * nchunks;
+  const float* pl = part_l + (long long)r * nchunks;
+  float M = -INFINITY;
+  for (int c = 0; c < nchunks; ++c) M = fmaxf(M, pm[c]);
+  float L = 0.f;
+  for (int c = 0; c < nchunks; ++c) {
+    if (pm[c] != -INFINITY) L += pl[c] * expf(pm[c] - M);
+  }
+  rowstat[2 * r] = M;
+  rowstat[2 * r + 1] = 1.0f / (L * (float)w);
+}
+
+__global__ void maxpool_kernel(const float* __restrict__ abar, float* __restrict__ attn, int n, int kp) {
+  const long long base = (long long)blockIdx.y * n;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int r = (kp - 1) / 2;
+  const int lo = max(i - r, 0), hi = min(i + r, n - 1);
+  float m = abar[base + lo];
+  for (int k = lo + 1; k <= hi; ++k) m = fmaxf(m, abar[base + k]);
+  attn[base + i] = m;
+}
+
+template <typename T, int DH, int WT>
+cudaError_t run(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, int* launches) {
+  const size_t smem = (size_t)(WT * DH + (kThreads / 32) * WT + 2 * WT) * sizeof(float);
+  auto k1 = attn_pass_kernel<T, DH, WT, false>;
+  auto k2 = attn_pass_kernel<T, DH, WT, true>;
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(k2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  dim3 grid(a.nchunks, d.Hq, d.nb);
+  k1<<<grid, kThreads, smem, st>>>(a);
+  const int rows = d.nb * d.Hq * d.w;
+  attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
+  k2<<<grid, kThreads, smem, st>>>(a);
+  dim3 pgrid((d.n + 255) / 256, d.nb * d.Hq);
+  maxpool_kernel<<<pgrid, 256, 0, st>>>(a.abar, attn, d.n, d.kp);
+  *launches += 4;
+  return cudaGetLastError();
+}
+
+template <typename T, int DH>
+cudaError_t run_w(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, int* launches) {
+  if (d.w <= 16) return run<T, DH, 16>(d, a, attn, st, launches);
+  if (d.w <= 32) return run<T, DH, 32>(d, a, attn, st, launches);
+  return run<T, DH, 64>(d, a, attn, st, launches);
+}
+
+}  // namespace
+
+cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K, float* attn,
+                                    const ScoreWorkspace& ws, cudaStream_t st, int* launches) {
+  AttnArgs a;
+  a.Qw = Qw; a.K = K;
+  a.part_m = ws.part_m; a.part_l = ws.part_l; a.rowstat = ws.rowstat; a.abar = ws.abar;
+  a.Hq = d.Hq; a.G = d.G; a.n = d.n; a.w = d.w;
+  a.nchunks = (d.n + kAttnChunk - 1) / kAttnChunk;
+  a.scale = d.scale;
+  for (int i = 0; i < 3; ++i) { a.qs[i] = d.qs[i]; a.ks[i] = d.ks[i]; }
+  if (d.dtype == CKV_F32) {
+    return d.dh == 64 ? run_w<float, 64>(d, a, attn, st, launches) : run_w<float, 128>(d, a, attn, st, launches);
+  }
+  return d.dh == 64 ? run_w<__nv_bfloat16, 64>(d, a, attn, st, launches)
+                    : run_w<__nv_bfloat16, 128>(d, a, attn, st, launches);
+}
+
+}  // namespace ckv
