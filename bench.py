@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the CriticalKV compression step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole path (window attention, projection norm, two-stage selection, gather) over a
+32-layer Llama-3.1-8B-shaped stack: 32 query heads / 8 KV heads, head_dim 128, d_model 4096, n = 32768 cached
+entries per head, window 32, pool kernel 7, flattened adaptive budget of 20% of the entries per layer; bf16 inputs,
+float32 scores.  Inputs are seeded synthetic tensors (gen/workloads.py).  With N > 1 (torchrun) every rank runs its
+own stack (independent layers, no collective on the data path): weak scaling.
+
+Prints one JSON line: whole-job KV entries scored+selected per second with inputs resident in HBM (`value`), the same
+through host buffers with the copies inside the timed region (`e2e`), the roofline of the dominant kernel (the
+projection-norm contraction, timed with CUDA events inside the timed region), and the CPU oracle timed on a bounded
+sample (`cpu_baseline`).  `--impl reference` times the CPU oracle alone.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "kv_entries_scored_selected_per_s"
+UNIT = "entries/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=5)
+    p.add_argument("--warmup", type=int, default=3)
+    p.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    p.add_argument("--cfg", type=int, default=3, help="workload id in gen.CONFIGS (3 = the headline 32-layer stack)")
+    p.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
+    p.add_argument("--no-cpu-baseline", action="store_true")
+    p.add_argument("--no-e2e", action="store_true")
+    return p.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            pk = json.load(f)
+        return pk, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = [ln for (t, ln) in self.lines if t0 <= t <= t1 + 0.2] or [ln for (_, ln) in self.lines]
+        for ln in rows:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax = float(parts[1])
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample(wl, layer=0):
+    """One full layer of the workload through the CPU oracle.  Returns (entries, seconds, threads)."""
+    from gen import make_layer
+    from oracle import criticalkv_oracle as oc
+    L = make_layer(wl, layer)
+    t0 = time.perf_counter()
+    oc.compress_layer(L.Qw, L.K, L.V, L.WO, kp=wl.kp, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha,
+                      eps=wl.eps, K_store=L.K_store, V_store=L.V_store)
+    dt = time.perf_counter() - t0
+    return wl.Hkv * wl.n, dt, len(os.sched_getaffinity(0))
+
+
+def run_reference(args, wl):
+    """The CPU oracle as the reference arm: each step is one full layer of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    times = []
+    for s in range(args.warmup + args.steps):
+        entries, dt, cores = oracle_sample(wl, layer=s % wl.layers)
+        if s >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = entries * len(times) / total
+    sample = f"1 of {wl.layers} layers per step (all heads, full n={wl.n}); numpy float64"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": wl.name, "note": "CPU oracle, one layer per step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    from gen import config, make_layer
+    wl = config(args.cfg)
+    if args.layers:
+        wl = wl.with_(layers=args.layers)
+    if args.impl == "reference":
+        run_reference(args, wl)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2502_03805_b200 import binding as B
+    from paper_2502_03805_b200 import session_for, to_device
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the compression path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.load()
+
+    nb = wl.layers
+    # every rank owns its own stack: layer seeds are offset by the rank
+    t_gen = time.time()
+    layers = [make_layer(wl, rank * nb + l) for l in range(nb)]
+    host = {}
+    for name in ("Qw_store", "K_store", "V_store", "WO_store"):
+        arr = np.stack([getattr(L, name) for L in layers])
+        t = torch.from_numpy(arr)
+        if wl.dtype == "bf16":
+            t = t.view(torch.bfloat16)
+        host[name] = t.pin_memory()
+    del layers
+    Qw, K, V, WO = (host[k].to(dev, non_blocking=True) for k in ("Qw_store", "K_store", "V_store", "WO_store"))
+    torch.cuda.synchronize()
+    t_gen = time.time() - t_gen
+
+    s = session_for(wl, nb=nb, device=local, want_stage=False)
+    stream = torch.cuda.current_stream()
+    gemm_ev = []
+
+    def step(record=False):
+        # the two halves of criticalkv_score are issued separately so that events can bracket the contraction
+        B.criticalkv_score(s.handle, s.desc, Qw, K, None, None, s.attn, None, s.ws, stream=stream)
+        if record:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+        B.criticalkv_score(s.handle, s.desc, None, None, V, WO, None, s.vnorm, s.ws, stream=stream)
+        if record:
+            e1.record(stream)
+            gemm_ev.append((e0, e1))
+        s.select(stream=stream)
+        s.compact(K, V, stream=stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = s.launches
+    barrier()
+    t0 = time.time()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(record=True)
+    ev1.record(stream)
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    launches = s.launches - launches0
+    assert s.device_status() == 0, "device status word set during the timed region"
+    ms_total = ev0.elapsed_time(ev1)
+    gemm_ms = [a.elapsed_time(b) for a, b in gemm_ev]
+    path = s.last_path
+
+    # ---- end to end: host buffers, copies inside the timed region, layer by layer on two streams ----
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, wl, host, local, world)
+
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total = float(t.item())
+    entries_per_step = world * nb * wl.Hkv * wl.n
+    ms_per_step = ms_total / args.steps
+    value = entries_per_step / (ms_per_step * 1e-3)
+
+    if rank == 0:
+        peaks, how = load_peaks()
+        flops = 2.0 * wl.n * wl.dh * wl.dm * wl.Hq * nb
+        gemm_avg = sum(gemm_ms) / len(gemm_ms)
+        achieved = flops / (gemm_avg * 1e-3) / 1e12
+        peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+        roofline = {"kernel": "projection norm (V W^O row L1 norm), step 2", "bound": "tensor",
+                    "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "peak_source": f"{how} (sustained bf16, kernel timed inside a long step)",
+                    "ms_per_launch": gemm_avg, "flops_per_launch": flops, "traffic": None,
+                    "tensor_core_path": bool(path & 2)}
+        cpu = None
+        if not args.no_cpu_baseline:
+            entries, dt, cores = oracle_sample(wl, 0)
+            cpu = {"value": entries / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"layer 0 of {wl.layers} (all heads, full n={wl.n}), {dt:.1f} s; numpy float64"}
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
+                "config": {"workload": wl.name, "layers": nb, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.dh,
+                           "d_model": wl.dm, "n": wl.n, "window": wl.w, "pool_kernel": wl.kp,
+                           "budget": f"{wl.budget_mode} {wl.budget} per layer", "alpha": wl.alpha,
+                           "l2": "inputs of one step (5.4 GB) exceed L2; layers are distinct buffers",
+                           "ms_per_32_layer_compression": ms_per_step * 32.0 / nb},
+                "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+                "cpu_baseline": cpu, "input_generation_s": round(t_gen, 1)}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, wl, host, local, world):
+    """Same metric with every step's inputs starting in pinned host memory and its results ending there.
+    Layers are streamed one at a time: copy-in, compress and copy-out of neighbouring layers overlap on two
+    streams with double-buffered device staging."""
+    import torch
+    import torch.distributed as dist
+    from paper_2502_03805_b200 import session_for
+    dev = torch.device("cuda", local)
+    nb = wl.layers
+    tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
+    sess = [session_for(wl, nb=1, device=local, want_stage=False) for _ in range(2)]
+    stage_in = [{k: torch.empty_like(v[0:1], device=dev) for k, v in host.items()} for _ in range(2)]
+    out_host = {"idx": torch.empty((nb, wl.btot), dtype=torch.int32).pin_memory(),
+                "offsets": torch.empty((nb, wl.Hkv + 1), dtype=torch.int32).pin_memory(),
+                "K_out": torch.empty((nb, wl.btot, wl.dh), dtype=tdt).pin_memory(),
+                "V_out": torch.empty((nb, wl.btot, wl.dh), dtype=tdt).pin_memory()}
+    streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
+    h2d = sum(v[0:1].numel() * v.element_size() for v in host.values()) * nb
+    d2h = sum(v[0:1].numel() * v.element_size() for v in out_host.values()) * nb
+
+    def step():
+        for l in range(nb):
+            p = l & 1
+            st, ss, si = streams[p], sess[p], stage_in[p]
+            with torch.cuda.stream(st):
+                for k in host:
+                    si[k].copy_(host[k][l:l + 1], non_blocking=True)
+                ss.compress(si["Qw_store"], si["K_store"], si["V_store"], si["WO_store"], stream=st)
+                out_host["idx"][l:l + 1].copy_(ss.idx, non_blocking=True)
+                out_host["offsets"][l:l + 1].copy_(ss.offsets, non_blocking=True)
+                out_host["K_out"][l:l + 1].copy_(ss.K_out, non_blocking=True)
+                out_host["V_out"][l:l + 1].copy_(ss.V_out, non_blocking=True)
+        for st in streams:
+            st.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(min(args.warmup, 2)):
+        step()
+    barrier()
+    steps = max(1, min(args.steps, 3))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        step()
+    barrier()
+    dt = time.perf_counter() - t0
+    t = torch.tensor([dt], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dt = float(t.item())
+    value = world * nb * wl.Hkv * wl.n * steps / dt
+    return {"value": value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+            "ms_per_step": 1e3 * dt / steps, "steps": steps,
+            "how": "per layer: pinned host -> device copies of Qw, K, V, W_O, criticalkv_compress, device -> pinned "
+                   "host copies of idx, offsets, K_out, V_out; two streams, double-buffered"}
+
+
+if __name__ == "__main__":
+    main()

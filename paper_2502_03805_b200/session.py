@@ -1,0 +1,99 @@
+"""Device-buffer plumbing around the C ABI: allocates outputs and workspace with torch and forwards to the binding.
+
+No step of the method runs here; every tensor is produced by the kernels of libcriticalkv.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+_TORCH_DTYPE = {"f32": torch.float32, "bf16": torch.bfloat16}
+
+
+def to_device(store: np.ndarray, dtype: str, device="cuda:0") -> torch.Tensor:
+    """Upload a stored array (float32, or uint16 bfloat16 bit patterns) without changing a bit."""
+    t = torch.from_numpy(np.ascontiguousarray(store))
+    if dtype == "bf16":
+        t = t.view(torch.bfloat16)
+    return t.to(device)
+
+
+def to_host(t: torch.Tensor) -> np.ndarray:
+    t = t.detach().cpu()
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).numpy().view(np.uint16)
+    return t.numpy()
+
+
+class CompressionSession:
+    """Holds a handle, a descriptor and the device buffers of one problem shape."""
+
+    def __init__(self, *, nb, Hq, Hkv, dh, dm, n, w, pool_k, dtype, budget_mode, budget, alpha=0.5, eps=1e-4,
+                 scale=0.0, flags=0, device=0, want_stage=True):
+        self.device = torch.device("cuda", device)
+        self.dtype = dtype
+        self.desc = B.make_desc(nb=nb, Hq=Hq, Hkv=Hkv, dh=dh, dm=dm, n=n, w=w, pool_k=pool_k, dtype=dtype,
+                                budget_mode=budget_mode, budget=budget, alpha=alpha, eps=eps, scale=scale,
+                                flags=flags)
+        self.handle = B.criticalkv_create(device)
+        self.btot = budget * Hkv if budget_mode == "uniform" else budget
+        sb, tb = B.criticalkv_workspace_bytes(self.desc)
+        dev = self.device
+        self.score_bytes, self.select_bytes = sb, tb
+        self.ws = torch.empty(max(sb, tb, 256), dtype=torch.uint8, device=dev)
+        self.attn = torch.empty((nb, Hq, n), dtype=torch.float32, device=dev)
+        self.vnorm = torch.empty((nb, Hq, n), dtype=torch.float32, device=dev)
+        self.idx = torch.full((nb, max(self.btot, 1)), -1, dtype=torch.int32, device=dev)
+        self.offsets = torch.zeros((nb, Hkv + 1), dtype=torch.int32, device=dev)
+        self.stage = torch.zeros((nb, max(self.btot, 1)), dtype=torch.uint8, device=dev) if want_stage else None
+        self.K_out = torch.zeros((nb, max(self.btot, 1), dh), dtype=_TORCH_DTYPE[dtype], device=dev)
+        self.V_out = torch.zeros_like(self.K_out)
+
+    def close(self):
+        if self.handle is not None:
+            B.criticalkv_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def score(self, Qw, K, V, WO, stream=None):
+        return B.criticalkv_score(self.handle, self.desc, Qw, K, V, WO, self.attn, self.vnorm, self.ws,
+                                  stream=stream)
+
+    def select(self, attn=None, vnorm=None, budgets_in=None, stream=None):
+        return B.criticalkv_select(self.handle, self.desc, self.attn if attn is None else attn,
+                                   self.vnorm if vnorm is None else vnorm, budgets_in, self.idx, self.offsets,
+                                   self.stage, self.ws, stream=stream)
+
+    def compact(self, K, V, stream=None):
+        return B.criticalkv_compact(self.handle, self.desc, K, V, self.idx, self.offsets, self.K_out, self.V_out,
+                                    stream=stream)
+
+    def compress(self, Qw, K, V, WO, budgets_in=None, stream=None):
+        return B.criticalkv_compress(self.handle, self.desc, Qw, K, V, WO, budgets_in, self.attn, self.vnorm,
+                                     self.idx, self.offsets, self.stage, self.K_out, self.V_out, self.ws,
+                                     stream=stream)
+
+    def device_status(self, stream=None):
+        return B.criticalkv_device_status(self.handle, stream)
+
+    @property
+    def launches(self):
+        return B.criticalkv_launch_count(self.handle)
+
+    @property
+    def last_path(self):
+        return B.criticalkv_last_path(self.handle)
+
+
+def session_for(wl, nb=1, **kw) -> CompressionSession:
+    """Session for a gen.Workload-like object (fields Hq, Hkv, dh, dm, n, w, kp, dtype, budget_mode, budget, ...)."""
+    return CompressionSession(nb=nb, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp,
+                              dtype=wl.dtype, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha,
+                              eps=wl.eps, **kw)

@@ -1,0 +1,175 @@
+"""GPU parity: the CUDA path (through the C ABI) against the CPU oracle on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from gen import config, make_layer, small_workload
+from oracle import criticalkv_oracle as oc
+
+import parity_util as pu
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(wl, layers=(0,), **kw):
+    from gpu_util import run_layers
+    Ls = [make_layer(wl, l) for l in layers]
+    outs, s = run_layers(Ls, wl, **kw)
+    return Ls, outs, s
+
+
+def test_config0_fp32_full_parity():
+    wl = config(0)
+    Ls, outs, s = _run(wl)
+    rep = pu.check_layer_against_oracle(Ls[0], wl, outs[0])
+    assert rep["attn_err"] < 1e-4 and rep["vnorm_err"] < 1e-4
+    assert s.launches > 0
+
+
+SMALL = [
+    dict(dtype="f32", n=300, w=8, kp=5, budget=40),                       # ragged tail in every tile size
+    dict(dtype="bf16", n=777, w=16, kp=7, budget=100, dh=128, dm=264),    # dm not a multiple of 64
+    dict(dtype="bf16", n=64, w=64, kp=3, budget=10, dh=64, dm=128, Hq=2, Hkv=2),   # n == w: pure causal window
+    dict(dtype="f32", n=33, w=1, kp=1, budget=5, Hq=2, Hkv=1),            # single query, no pooling
+    dict(dtype="bf16", n=1000, w=32, kp=7, budget=1000, dh=128, dm=256),  # keep everything
+    dict(dtype="bf16", n=513, w=32, kp=7, budget=0, dh=128, dm=256),      # keep nothing
+    dict(dtype="f32", n=257, w=16, kp=9, budget=1, dh=64, dm=64),         # b' = 0, b'' = 1
+    dict(dtype="bf16", n=2049, w=33, kp=7, budget=300, dh=128, dm=512, Hq=10, Hkv=2),   # group of 5, odd window
+    dict(dtype="bf16", n=1500, w=32, kp=7, budget_mode="adaptive", budget=700, dh=128, dm=256, Hq=8, Hkv=4),
+    dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=0.25),
+    dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=1.0),
+    dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=0.0),
+]
+
+
+@pytest.mark.parametrize("case", range(len(SMALL)))
+def test_small_and_edge_cases(case):
+    wl = small_workload(cfg_id=100 + case, **SMALL[case])
+    Ls, outs, _ = _run(wl, layers=(0, 1))
+    for L, out in zip(Ls, outs):
+        pu.check_layer_against_oracle(L, wl, out)
+
+
+def test_separate_calls_equal_fused_call_and_are_deterministic():
+    wl = small_workload(cfg_id=130, dtype="bf16", n=900, w=32, kp=7, budget=120, dh=128, dm=256)
+    _, a, _ = _run(wl)
+    _, b, _ = _run(wl, separate_calls=True)
+    _, c, _ = _run(wl)
+    for k in a[0]:
+        np.testing.assert_array_equal(a[0][k], b[0][k])
+        np.testing.assert_array_equal(a[0][k], c[0][k])
+
+
+def _select_on_given_scores(P, nu, wl, budgets_in=None):
+    from paper_2502_03805_b200 import session_for
+    s = session_for(wl, nb=1)
+    attn = torch.from_numpy(P.astype(np.float32))[None].cuda()
+    vnorm = torch.from_numpy(nu.astype(np.float32))[None].cuda()
+    bi = None if budgets_in is None else torch.tensor(budgets_in, dtype=torch.int32, device="cuda")[None]
+    s.select(attn, vnorm, budgets_in=bi)
+    torch.cuda.synchronize()
+    return s.idx[0].cpu().numpy(), s.offsets[0].cpu().numpy(), s.stage[0].cpu().numpy(), s
+
+
+@pytest.mark.parametrize("mode,budget", [("uniform", 97), ("adaptive", 500), ("uniform", 0), ("adaptive", 4 * 1237)])
+@pytest.mark.parametrize("ties", [False, True])
+def test_select_is_bit_exact_on_identical_scores(mode, budget, ties):
+    # same float32 scores on both sides: the integer decisions must agree exactly, ties included
+    r = np.random.default_rng(5)
+    Hq, Hkv, n = 12, 4, 1237
+    P = r.random((Hq, n)).astype(np.float32) ** 8
+    nu = np.exp(r.standard_normal((Hq, n))).astype(np.float32)
+    if ties:
+        P = (np.round(P * 8) / 8).astype(np.float32)          # long runs of equal scores, as pooling produces
+        nu = np.round(nu).astype(np.float32)
+    wl = small_workload(cfg_id=140, Hq=Hq, Hkv=Hkv, n=n, budget_mode=mode, budget=budget)
+    ref = oc.select(P, nu, G=3, budget_mode=mode, budget=budget, alpha=0.5, eps=1e-4)
+    idx, off, st, _ = _select_on_given_scores(P, nu, wl)
+    np.testing.assert_array_equal(off, ref["offsets"])
+    tot = ref["offsets"][-1]
+    np.testing.assert_array_equal(idx[:tot], ref["idx"])
+    np.testing.assert_array_equal(st[:tot], ref["stage"])
+
+
+def test_select_given_budgets():
+    r = np.random.default_rng(6)
+    Hq, Hkv, n = 4, 4, 640
+    P = r.random((Hq, n)).astype(np.float32)
+    nu = r.random((Hq, n)).astype(np.float32)
+    budgets = [0, 640, 17, 100]
+    wl = small_workload(cfg_id=141, Hq=Hq, Hkv=Hkv, n=n, budget_mode="given", budget=800)
+    ref = oc.select(P, nu, G=1, budget_mode="given", budget=800, budgets_in=budgets)
+    idx, off, st, s = _select_on_given_scores(P, nu, wl, budgets)
+    np.testing.assert_array_equal(off, ref["offsets"])
+    np.testing.assert_array_equal(idx[: off[-1]], ref["idx"])
+    assert s.device_status() == 0
+    # budgets beyond the capacity are clipped and reported, never written out of bounds
+    idx2, off2, _, s2 = _select_on_given_scores(P, nu, wl, [640, 640, 0, 0])
+    assert off2[-1] <= 800 and s2.device_status() != 0
+
+
+def test_strided_kv_layout():
+    # K/V stored token-major [n, Hkv, dh] and addressed through the descriptor's strides
+    from paper_2502_03805_b200 import CompressionSession, to_device, to_host
+    wl = small_workload(cfg_id=150, dtype="bf16", n=600, w=16, kp=5, budget=64, dh=128, dm=256)
+    L = make_layer(wl)
+    Kt = np.ascontiguousarray(L.K_store.transpose(1, 0, 2))
+    Vt = np.ascontiguousarray(L.V_store.transpose(1, 0, 2))
+    s = CompressionSession(nb=1, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp,
+                           dtype="bf16", budget_mode="uniform", budget=wl.budget)
+    s.desc.k_stride[:] = (wl.n * wl.Hkv * wl.dh, wl.dh, wl.Hkv * wl.dh)
+    s.desc.v_stride[:] = (wl.n * wl.Hkv * wl.dh, wl.dh, wl.Hkv * wl.dh)
+    K, V = to_device(Kt, "bf16"), to_device(Vt, "bf16")
+    s.compress(to_device(L.Qw_store[None], "bf16"), K, V, to_device(L.WO_store[None], "bf16"))
+    torch.cuda.synchronize()
+    out = dict(attn=to_host(s.attn[0]), vnorm=to_host(s.vnorm[0]), idx=to_host(s.idx[0]),
+               offsets=to_host(s.offsets[0]), stage=to_host(s.stage[0]), K_out=to_host(s.K_out[0]),
+               V_out=to_host(s.V_out[0]))
+    pu.check_layer_against_oracle(L, wl, out)
+
+
+def test_config1_full_parity():
+    wl = config(1)
+    Ls, outs, _ = _run(wl)
+    rep = pu.check_layer_against_oracle(Ls[0], wl, outs[0])
+    print("config1", rep)
+
+
+def test_config2_full_parity():
+    wl = config(2)
+    Ls, outs, _ = _run(wl)
+    rep = pu.check_layer_against_oracle(Ls[0], wl, outs[0], full_output_check=True)
+    print("config2", rep)
+
+
+def test_config3_two_layers_adaptive_parity():
+    # the sparsest and the densest attention of the 32 layers (by the recipe's per-layer concentration target)
+    wl = config(3)
+    shares = [make_layer(wl.with_(n=64, dm=8), l).share_target for l in range(wl.layers)]
+    layers = (int(np.argmin(shares)), int(np.argmax(shares)))
+    Ls, outs, _ = _run(wl, layers=layers)
+    for L, out in zip(Ls, outs):
+        rep = pu.check_layer_against_oracle(L, wl, out)
+        print("config3 layer", L.layer, rep)
+
+
+@pytest.mark.parametrize("mode", ["uniform", "adaptive"])
+def test_config4_one_layer_sampled(mode):
+    # n = 131072: attention compared in full, the projection norm on 4096 sampled rows per head, and the selection
+    # against the oracle's rule applied to the GPU's own float32 scores (bit-exact by construction of the rule)
+    wl = config(4)
+    if mode == "adaptive":
+        wl = wl.with_(budget_mode="adaptive", budget=8 * wl.budget)
+    Ls, outs, _ = _run(wl)
+    L, out = Ls[0], outs[0]
+    P = oc.pooled_window_attention(L.Qw, L.K, wl.kp, wl.scale)
+    pu.assert_scores_close(out["attn"], P, "attn")
+    rows = np.sort(np.random.default_rng(4).choice(wl.n, 4096, replace=False))
+    nu = oc.projection_norm(L.V, L.WO, rows=rows)
+    pu.assert_scores_close(out["vnorm"][:, rows], nu, "vnorm (sampled rows)")
+    ref = oc.select(out["attn"], out["vnorm"], G=wl.G, budget_mode=wl.budget_mode, budget=wl.budget,
+                    alpha=wl.alpha, eps=wl.eps)
+    np.testing.assert_array_equal(out["offsets"], ref["offsets"])
+    np.testing.assert_array_equal(out["idx"][: ref["idx"].size], ref["idx"])
+    np.testing.assert_array_equal(out["stage"][: ref["idx"].size], ref["stage"])
+    pu.assert_compaction_exact(L.K_store, L.V_store, out["idx"], out["offsets"], out["K_out"], out["V_out"])
