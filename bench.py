@@ -159,7 +159,8 @@ def main():
     import torch
     import torch.distributed as dist
     from paper_2502_03805_b200 import binding as B
-    from paper_2502_03805_b200 import session_for, to_device
+    from paper_2502_03805_b200 import session_for
+    from paper_2502_03805_b200.dist_util import max_over_ranks, rank_layer_ids, whole_job_throughput
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -175,7 +176,7 @@ def main():
     nb = wl.layers
     # every rank owns its own stack: layer seeds are offset by the rank
     t_gen = time.time()
-    layers = [make_layer(wl, rank * nb + l) for l in range(nb)]
+    layers = [make_layer(wl, l) for l in rank_layer_ids(rank, nb)]
     host = {}
     for name in ("Qw_store", "K_store", "V_store", "WO_store"):
         arr = np.stack([getattr(L, name) for L in layers])
@@ -238,13 +239,9 @@ def main():
     if not args.no_e2e:
         e2e = run_e2e(args, wl, host, local, world)
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
-    entries_per_step = world * nb * wl.Hkv * wl.n
+    ms_total = max_over_ranks(ms_total, dev)
     ms_per_step = ms_total / args.steps
-    value = entries_per_step / (ms_per_step * 1e-3)
+    value = whole_job_throughput(nb * wl.Hkv * wl.n, world, ms_per_step * 1e-3)
 
     if rank == 0:
         peaks, how = load_peaks()
@@ -326,11 +323,9 @@ def run_e2e(args, wl, host, local, world):
         step()
     barrier()
     dt = time.perf_counter() - t0
-    t = torch.tensor([dt], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dt = float(t.item())
-    value = world * nb * wl.Hkv * wl.n * steps / dt
+    from paper_2502_03805_b200.dist_util import max_over_ranks, whole_job_throughput
+    dt = max_over_ranks(dt, dev)
+    value = whole_job_throughput(nb * wl.Hkv * wl.n * steps, world, dt)
     return {"value": value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
             "ms_per_step": 1e3 * dt / steps, "steps": steps,
             "how": "per layer: pinned host -> device copies of Qw, K, V, W_O, criticalkv_compress, device -> pinned "

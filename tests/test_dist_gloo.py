@@ -1,0 +1,46 @@
+"""World-size-2 CPU test (gloo) of the multi-rank bookkeeping used by bench.py --gpus N."""
+import os
+import socket
+
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+from paper_2502_03805_b200.dist_util import max_over_ranks, rank_layer_ids, whole_job_throughput
+
+
+def _free_port():
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    local_ms = 10.0 + 5.0 * rank                      # rank 1 is the slow one
+    slowest = max_over_ranks(local_ms)
+    dist.barrier()
+    out.put((rank, slowest, rank_layer_ids(rank, 4)))
+    dist.destroy_process_group()
+
+
+def test_two_ranks_take_the_max_time_and_own_disjoint_layers():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [r[1] for r in res] == [15.0, 15.0]
+    assert res[0][2] == [0, 1, 2, 3] and res[1][2] == [4, 5, 6, 7]
+    assert whole_job_throughput(1000, 2, 0.015) == 2000 / 0.015
+
+
+def test_single_process_is_identity():
+    assert max_over_ranks(3.5) == 3.5
