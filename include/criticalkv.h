@@ -125,6 +125,28 @@ CKV_API int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, con
                               const int32_t* budgets_in, int32_t* idx, int32_t* offsets, uint8_t* stage, void* ws,
                               size_t ws_bytes, void* stream);
 
+/*
+ * Allocation-free variant of criticalkv_select (the paper has no counterpart: this is a packaging of steps 3-4 for
+ * callers that cannot provide a workspace).  Some hosts of this library may not allocate device memory at the point
+ * where they compress a cache: a serving engine that reserved all of HBM for its own pools at start-up has nothing
+ * left for cudaMalloc, and a latency-critical loop cannot afford the device-wide synchronisation an allocation or a
+ * free implies.  This entry point therefore takes no workspace: the group scores and per-head budgets go to a fixed
+ * array of CKV_STATIC_SCRATCH_BYTES that lives inside the library image (every GPU that loads the library keeps
+ * that much memory until the process exits).  Arguments and results are those of criticalkv_select.
+ *   - The request must fit: if the select_bytes that criticalkv_workspace_bytes reports exceeds
+ *     CKV_STATIC_SCRATCH_BYTES (about nb*Hkv*n > 2^20 scored entries) the call returns CKV_EWORKSPACE, launches
+ *     nothing, and criticalkv_last_cuda_error describes the sizes.
+ *   - The first call on each device looks up the array's device address (once, with that device current); make that
+ *     first call outside any stream capture.  No call allocates or frees device memory.
+ *   - All calls, from every handle and stream of the process, share the one array per device.  Nothing is read from
+ *     it before this call has written it, so stale contents are harmless, but two calls whose kernels may overlap on
+ *     the GPU (different streams) race on it: order them on one stream or with events.
+ */
+#define CKV_STATIC_SCRATCH_BYTES ((size_t)((8u << 20) + (64u << 10)))
+CKV_API int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc* d, const float* attn,
+                                     const float* vnorm, const int32_t* budgets_in, int32_t* idx, int32_t* offsets,
+                                     uint8_t* stage, void* stream);
+
 /* Step 5.  K_out[nb, r, :] = K[nb, g, idx[nb, r], :] for r in head g's segment, same for V (bit copy). */
 CKV_API int criticalkv_compact(criticalkv_handle h, const criticalkv_desc* d, const void* K, const void* V,
                                const int32_t* idx, const int32_t* offsets, void* K_out, void* V_out, void* stream);
@@ -139,7 +161,8 @@ CKV_API int criticalkv_compress(criticalkv_handle h, const criticalkv_desc* d, c
 CKV_API int criticalkv_device_status(criticalkv_handle h, void* stream, int* out);
 
 CKV_API const char* criticalkv_status_string(int status);
-/* Last CUDA error string seen by this handle ("" if none); valid until the next call on the handle. */
+/* Last CUDA error string (or size diagnostic of criticalkv_select_static) seen by this handle ("" if none); valid
+   until the next call on the handle. */
 CKV_API const char* criticalkv_last_cuda_error(criticalkv_handle h);
 /* Which kernels the last criticalkv_score on this handle launched: bit0 tensor-core window attention,
    bit1 tensor-core projection norm, bit2 CUDA-core window attention, bit3 CUDA-core projection norm. */

@@ -17,9 +17,10 @@ CKV_F32, CKV_BF16 = 0, 1
 CKV_BUDGET_UNIFORM, CKV_BUDGET_FLAT_ADAPTIVE, CKV_BUDGET_GIVEN = 0, 1, 2
 CKV_NORM_L1 = 0
 CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT = 1, 2
+CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",
-           "criticalkv_select", "criticalkv_compact", "criticalkv_compress", "criticalkv_device_status",
+           "criticalkv_select", "criticalkv_select_static", "criticalkv_compact", "criticalkv_compress", "criticalkv_device_status",
            "criticalkv_status_string", "criticalkv_last_cuda_error", "criticalkv_last_path",
            "criticalkv_launch_count")
 
@@ -59,6 +60,7 @@ def load():
     lib.criticalkv_workspace_bytes.argtypes = [dp, C.POINTER(sz), C.POINTER(sz)]
     lib.criticalkv_score.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.criticalkv_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.criticalkv_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
     lib.criticalkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
     lib.criticalkv_compress.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.criticalkv_device_status.argtypes = [vp, vp, C.POINTER(i32)]
@@ -155,6 +157,16 @@ def criticalkv_select(handle, desc, attn, vnorm, budgets_in, idx, offsets, stage
     rc = load().criticalkv_select(handle, C.byref(desc), _ptr(attn), _ptr(vnorm), _ptr(budgets_in), _ptr(idx),
                                   _ptr(offsets), _ptr(stage), _ptr(ws), _nbytes(ws, ws_bytes), _stream(stream))
     return _check(handle, rc, "criticalkv_select", check)
+
+
+def criticalkv_select_static(handle, desc, attn, vnorm, budgets_in, idx, offsets, stage, stream=None, check=True):
+    """criticalkv_select without a workspace argument: the scratch is a fixed array inside the library, for callers
+    that cannot allocate device memory when they compress (memory fully handed to their own pools, or a loop that
+    must not hit the synchronisation an allocation implies).  Shapes whose select workspace exceeds
+    CKV_STATIC_SCRATCH_BYTES are refused with CKV_EWORKSPACE; calls share the array, so do not let two overlap."""
+    rc = load().criticalkv_select_static(handle, C.byref(desc), _ptr(attn), _ptr(vnorm), _ptr(budgets_in), _ptr(idx),
+                                         _ptr(offsets), _ptr(stage), _stream(stream))
+    return _check(handle, rc, "criticalkv_select_static", check)
 
 
 def criticalkv_compact(handle, desc, K, V, idx, offsets, K_out, V_out, stream=None, check=True):

@@ -4,6 +4,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 
 #include "ckv_internal.h"
@@ -275,6 +276,65 @@ int criticalkv_device_status(criticalkv_handle h, void* stream, int* out) {
   if (e == cudaSuccess) e = cudaMemsetAsync(h->status_word, 0, sizeof(int), st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(st);
   *out = v;
+  return record_cuda(h, e);
+}
+
+// ---- allocation-free select ------------------------------------------------------------------------------------
+// Scratch for criticalkv_select_static.  The symbol below is only a stand-in on the host: kernels must be given the
+// device address that cudaGetSymbolAddress returns for the current device, never the name itself.
+}  // extern "C"
+static __device__ __align__(256) unsigned char g_select_static_scratch[CKV_STATIC_SCRATCH_BYTES];
+namespace {
+constexpr int kMaxStaticDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_scratch_addr[kMaxStaticDevices];  // per device ordinal, resolved on first use
+
+// Device address of the scratch array on `device` (which must be current).  Looked up once per device.
+cudaError_t static_scratch_address(int device, void** out) {
+  if (device < 0 || device >= kMaxStaticDevices) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (!g_static_scratch_addr[device]) {
+    void* p = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&p, g_select_static_scratch);
+    if (e != cudaSuccess) return e;
+    g_static_scratch_addr[device] = p;
+  }
+  *out = g_static_scratch_addr[device];
+  return cudaSuccess;
+}
+}  // namespace
+extern "C" {
+
+int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc* d, const float* attn, const float* vnorm,
+                             const int32_t* budgets_in, int32_t* idx, int32_t* offsets, uint8_t* stage,
+                             void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (!attn || !vnorm || !idx || !offsets) return CKV_EINVAL;
+  if (dd.budget_mode == CKV_BUDGET_GIVEN && !budgets_in) return CKV_EINVAL;
+  if (!aligned16(attn) || !aligned16(vnorm) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
+      (reinterpret_cast<uintptr_t>(offsets) & 3u) || (reinterpret_cast<uintptr_t>(budgets_in) & 3u))
+    return CKV_EALIGN;
+  const SelectLayout L = select_layout(dd);
+  if (L.total > CKV_STATIC_SCRATCH_BYTES) {
+    snprintf(h->cuda_error, sizeof(h->cuda_error),
+             "criticalkv_select_static: this shape needs %zu bytes of scratch, the built-in array holds %zu",
+             L.total, (size_t)CKV_STATIC_SCRATCH_BYTES);
+    return CKV_EWORKSPACE;
+  }
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  void* scratch = nullptr;
+  cudaError_t e = static_scratch_address(h->device, &scratch);
+  if (e != cudaSuccess) return record_cuda(h, e);
+  char* base = (char*)scratch;
+  ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets)};
+  int launches = 0;
+  e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, (cudaStream_t)stream, &launches,
+                         h->status_word);
+  h->launches += launches;
   return record_cuda(h, e);
 }
 
