@@ -201,8 +201,20 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
     path |= 4;
   }
   if (e == cudaSuccess && vnorm) {
-    e = ckv::launch_vnorm_simt(dd, V, WO, vnorm, st, &launches);
-    path |= 8;
+    bool done = false;
+    if (dd.dtype == CKV_BF16 && !(d->flags & CKV_FLAG_FORCE_SIMT) && h->cc_major == 10) {
+      e = ckv::launch_vnorm_umma(dd, V, WO, vnorm, h->sm_count, h->status_word, st, &launches);
+      if (e == cudaSuccess) {
+        done = true;
+        path |= 2;
+      } else if (e == cudaErrorNotSupported) {
+        e = cudaSuccess;
+      }
+    }
+    if (!done && e == cudaSuccess) {
+      e = ckv::launch_vnorm_simt(dd, V, WO, vnorm, st, &launches);
+      path |= 8;
+    }
   }
   h->launches += launches;
   h->last_path = path;

@@ -40,6 +40,10 @@ cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K
                                     const ScoreWorkspace& ws, cudaStream_t st, int* launches);
 cudaError_t launch_vnorm_simt(const Dims& d, const void* V, const void* WO, float* vnorm, cudaStream_t st,
                               int* launches);
+// Tensor-core projection norm (bf16).  cudaErrorNotSupported = this layout cannot be expressed as a tensor map;
+// the caller then uses the CUDA-core kernel.
+cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, float* vnorm, int sm_count,
+                              int* status_word, cudaStream_t st, int* launches);
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word);
