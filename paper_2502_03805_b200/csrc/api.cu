@@ -92,7 +92,9 @@ struct ScoreLayout {
 ScoreLayout score_layout(const Dims& d) {
   ScoreLayout L;
   const size_t rows = (size_t)d.nb * d.Hq * d.w;
-  const size_t nchunks = (d.n + ckv::kAttnChunk - 1) / ckv::kAttnChunk;
+  // one partial per 256 keys on the CUDA-core path; the tensor-core path writes two per work item of at least
+  // four 128-key tiles, the last item of a head possibly shorter: never more than ceil(n / 256) + 2
+  const size_t nchunks = (d.n + ckv::kAttnChunk - 1) / ckv::kAttnChunk + 2;
   size_t off = 0;
   L.part_m = off; off = align_up(off + rows * nchunks * sizeof(float), 256);
   L.part_l = off; off = align_up(off + rows * nchunks * sizeof(float), 256);
@@ -197,8 +199,20 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
   int launches = 0, path = 0;
   cudaError_t e = cudaSuccess;
   if (attn) {
-    e = ckv::launch_window_attn_simt(dd, Qw, K, attn, sw, st, &launches);
-    path |= 4;
+    bool done = false;
+    if (dd.dtype == CKV_BF16 && !(d->flags & CKV_FLAG_FORCE_SIMT) && h->cc_major == 10) {
+      e = ckv::launch_window_attn_umma(dd, Qw, K, attn, sw, h->sm_count, h->status_word, st, &launches);
+      if (e == cudaSuccess) {
+        done = true;
+        path |= 1;
+      } else if (e == cudaErrorNotSupported) {
+        e = cudaSuccess;
+      }
+    }
+    if (!done && e == cudaSuccess) {
+      e = ckv::launch_window_attn_simt(dd, Qw, K, attn, sw, st, &launches);
+      path |= 4;
+    }
   }
   if (e == cudaSuccess && vnorm) {
     bool done = false;

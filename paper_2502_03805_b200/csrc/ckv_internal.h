@@ -40,6 +40,14 @@ cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K
                                     const ScoreWorkspace& ws, cudaStream_t st, int* launches);
 cudaError_t launch_vnorm_simt(const Dims& d, const void* V, const void* WO, float* vnorm, cudaStream_t st,
                               int* launches);
+// Pieces of the window-attention path shared by the CUDA-core and tensor-core front ends.
+cudaError_t launch_attn_combine(const float* part_m, const float* part_l, float* rowstat, int rows, int nchunks,
+                                int w, cudaStream_t st);
+cudaError_t launch_maxpool(const float* abar, float* attn, int n, int kp, int nrows, cudaStream_t st);
+// Tensor-core window attention (bf16).  cudaErrorNotSupported = shape or layout outside what it handles.
+cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K, float* attn,
+                                    const ScoreWorkspace& ws, int sm_count, int* status_word, cudaStream_t st,
+                                    int* launches);
 // Tensor-core projection norm (bf16).  cudaErrorNotSupported = this layout cannot be expressed as a tensor map;
 // the caller then uses the CUDA-core kernel.
 cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, float* vnorm, int sm_count,

@@ -19,6 +19,7 @@
 
 #include "ckv_internal.h"
 #include "sm100_ptx.cuh"
+#include "tma_host.h"
 
 namespace ckv {
 namespace {
@@ -285,41 +286,6 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
   }
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
-  return fn;
-}
-
-// 4-D bf16 tensor map with a [box0 x box1 x 1 x 1] box and 128-byte swizzle.  Strides in elements for dims 1..3.
-bool make_map(CUtensorMap* m, const void* base, const cuuint64_t dims[4], const long long strides_elems[3],
-              cuuint32_t box0, cuuint32_t box1) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t gstr[3];
-  for (int i = 0; i < 3; ++i) {
-    gstr[i] = (cuuint64_t)strides_elems[i] * 2;
-    if (gstr[i] % 16 != 0 || gstr[i] >= (1ull << 40)) return false;
-  }
-  const cuuint32_t box[4] = {box0, box1, 1, 1};
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, gstr, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int DH>
 cudaError_t run(const Dims& d, const CUtensorMap& mv, const CUtensorMap& mw, const UmmaArgs& a, int sm_count,
                 cudaStream_t st) {
@@ -336,7 +302,7 @@ cudaError_t run(const Dims& d, const CUtensorMap& mv, const CUtensorMap& mw, con
 }  // namespace
 
 bool vnorm_umma_supported(const Dims& d) {
-  return d.dtype == CKV_BF16 && (d.dh == 64 || d.dh == 128) && d.vs[2] >= d.dh && encode_fn() != nullptr;
+  return d.dtype == CKV_BF16 && (d.dh == 64 || d.dh == 128) && d.vs[2] >= d.dh && tma_encode_fn() != nullptr;
 }
 
 // Returns cudaErrorNotSupported when the tensor maps cannot be encoded for this layout (caller falls back to the
@@ -347,11 +313,13 @@ cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, floa
   CUtensorMap mv, mw;
   const cuuint64_t vdims[4] = {(cuuint64_t)d.dh, (cuuint64_t)d.n, (cuuint64_t)d.Hkv, (cuuint64_t)d.nb};
   const long long vstr[3] = {d.vs[2], d.vs[1], d.vs[0]};
-  if (!make_map(&mv, V, vdims, vstr, 64, 128)) return cudaErrorNotSupported;
+  const cuuint32_t vbox[4] = {64, 128, 1, 1};
+  if (!make_bf16_map_4d(&mv, V, vdims, vstr, vbox)) return cudaErrorNotSupported;
   const int nbw = d.wo_shared ? 1 : d.nb;
   const cuuint64_t wdims[4] = {(cuuint64_t)d.dm, (cuuint64_t)d.dh, (cuuint64_t)d.Hq, (cuuint64_t)nbw};
   const long long wstr[3] = {d.dm, (long long)d.dh * d.dm, (long long)d.Hq * d.dh * d.dm};
-  if (!make_map(&mw, WO, wdims, wstr, 64, (cuuint32_t)d.dh)) return cudaErrorNotSupported;
+  const cuuint32_t wbox[4] = {64, (cuuint32_t)d.dh, 1, 1};
+  if (!make_bf16_map_4d(&mw, WO, wdims, wstr, wbox)) return cudaErrorNotSupported;
   UmmaArgs a;
   a.vnorm = vnorm; a.status = status_word;
   a.Hq = d.Hq; a.Hkv = d.Hkv; a.G = d.G; a.n = d.n; a.dm = d.dm; a.nb = d.nb;

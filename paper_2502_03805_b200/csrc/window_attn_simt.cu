@@ -228,6 +228,18 @@ cudaError_t run_w(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st
 
 }  // namespace
 
+cudaError_t launch_attn_combine(const float* part_m, const float* part_l, float* rowstat, int rows, int nchunks,
+                                int w, cudaStream_t st) {
+  attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(part_m, part_l, rowstat, rows, nchunks, w);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_maxpool(const float* abar, float* attn, int n, int kp, int nrows, cudaStream_t st) {
+  dim3 pgrid((n + 255) / 256, nrows);
+  maxpool_kernel<<<pgrid, 256, 0, st>>>(abar, attn, n, kp);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K, float* attn,
                                     const ScoreWorkspace& ws, cudaStream_t st, int* launches) {
   AttnArgs a;

@@ -1,0 +1,481 @@
+// Step 1 on the tensor cores (bf16): observation-window attention of Algorithm 2 (softmax and scale as in Eq. 2).
+//
+// The logits of a KV group (G query heads x w window rows, e.g. 4 x 32 = 128 rows) against a tile of 128 keys are one
+// tcgen05 MMA shape, so QK^T runs on the tensor cores and the K stream stays memory-bound.  Softmax needs every row's
+// maximum and sum before any weight can be normalised, hence two sweeps over K (the second is served from L2 when the
+// working set allows):
+//   sweep 1 (kStats) : D = Q_g K_tile^T, rows = query rows.  A thread owns one query row, keeps its running (max, sum)
+//                      over the key columns it reads from tensor memory, and stores one partial per work item.
+//                      The partials are merged by the same combine kernel the CUDA-core path uses.
+//   sweep 2 (kProbs) : D = K_tile Q_g^T, rows = keys.  A thread owns one key and sums the normalised weights of the w
+//                      window rows of each head straight from its tensor-memory lane: the window mean comes out
+//                      without any cross-lane traffic and is written coalesced along the sequence.
+// Max-pooling runs afterwards in the shared pooling kernel.
+//
+// Persistent kernel, one CTA per SM: warp 0 streams K tiles (and the group's Q rows, once per work item) with TMA,
+// warp 1 issues the MMAs, warps 2-9 are two sets of four softmax warps that take alternating accumulators (two
+// 256-column TMEM slots), so that the exponentials of one tile overlap the MMAs and TMEM loads of the next.
+// All waits are bounded (status word CKV_ETIMEOUT, tensor memory freed, normal return).
+#include <cuda_bf16.h>
+#include <math.h>
+
+#include "ckv_internal.h"
+#include "sm100_ptx.cuh"
+#include "tma_host.h"
+
+namespace ckv {
+namespace {
+
+using namespace ptx;
+
+constexpr int kKeyTile = 128;
+constexpr int kThreads = 10 * 32;
+constexpr int kSlotCols = 256;
+constexpr int kMaxRowBlocks = 3;  // G*w <= 384
+constexpr float kLog2e = 1.4426950408889634f;
+
+enum { kStats = 1, kProbs = 2 };
+
+struct AttnUmmaArgs {
+  float* part_m;
+  float* part_l;
+  const float* rowstat;
+  float* abar;
+  int* status;
+  int Hq, Hkv, G, n, nb;
+  int rows;            // G * w
+  int row_blocks;      // ceil(rows / 128)                          (sweep 1 sub-tiles per key tile)
+  int heads_per_group; // heads per MMA in sweep 2 (hg * w <= 256)
+  int head_groups;     // ceil(G / heads_per_group)                 (sweep 2 sub-tiles per key tile)
+  int ntiles;          // ceil(n / 128)
+  int tiles_per_item;
+  int chunks_per_bg;   // work items per (nb, KV head)
+  int part_stride;     // partial slots per row = 2 * chunks_per_bg
+  int kstages;
+  int qbufs;           // 1 or 2 shared-memory copies of the group's Q rows (and statistics)
+  float c;             // scale * log2(e)
+  float scale;
+  long long nitems;
+};
+
+struct Item {
+  int b, g, chunk, t0, t1;
+};
+__device__ __forceinline__ Item decode_item(long long item, const AttnUmmaArgs& a) {
+  Item it;
+  it.chunk = (int)(item % a.chunks_per_bg);
+  const long long r = item / a.chunks_per_bg;
+  it.g = (int)(r % a.Hkv);
+  it.b = (int)(r / a.Hkv);
+  it.t0 = it.chunk * a.tiles_per_item;
+  it.t1 = min(it.t0 + a.tiles_per_item, a.ntiles);
+  return it;
+}
+
+// Shared-memory carve-up (byte offsets from the 1024-aligned base).
+template <int DH>
+struct Layout {
+  int q_panel;   // bytes between the 64-element K panels of the Q rows
+  int q_bytes;
+  int k_off, k_stage;
+  int stats_off;  // two buffers of rows * 8 bytes
+  int bar_off;
+  int total;
+  __host__ __device__ Layout(int rows, int kstages, int qbufs) {
+    q_panel = rows * 128;
+    q_bytes = (q_panel * (DH / 64) + 1023) / 1024 * 1024;
+    k_off = qbufs * q_bytes;
+    k_stage = kKeyTile * DH * 2;
+    stats_off = k_off + kstages * k_stage;
+    bar_off = stats_off + 2 * rows * 8;
+    bar_off = (bar_off + 15) / 16 * 16;
+    total = bar_off + 25 * 8 + 16;
+  }
+};
+
+template <int DH, int W, int PASS>
+__global__ void __launch_bounds__(kThreads, 1)
+window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                        AttnUmmaArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const Layout<DH> L(a.rows, a.kstages, a.qbufs);
+  const uint32_t sbase = smem_addr(smem);
+  const uint32_t bars = sbase + L.bar_off;
+  auto q_full = [&](int s) { return bars + 8u * s; };
+  auto q_empty = [&](int s) { return bars + 8u * (2 + s); };
+  auto k_full = [&](int s) { return bars + 8u * (4 + s); };
+  auto k_empty = [&](int s) { return bars + 8u * (12 + s); };
+  auto t_full = [&](int s) { return bars + 8u * (20 + s); };
+  auto t_empty = [&](int s) { return bars + 8u * (22 + s); };
+  const uint32_t drain_bar = bars + 8u * 24;
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + 25 * 8);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+  volatile uint32_t* never = tmem_slot + 2;
+  float2* stats = reinterpret_cast<float2*>(smem + L.stats_off);  // [2][rows]: (-max * log2e, 1 / (w * sum))
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  constexpr int kKSteps = DH / 16;
+  constexpr int kPanels = DH / 64;
+  const int nsub = PASS == kStats ? a.row_blocks : a.head_groups;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(q_full(s), 1);
+      // a Q buffer is free again when the MMAs of its item have retired and, in the second sweep, when all eight
+      // softmax warps are done with the item's statistics
+      mbar_init(q_empty(s), PASS == kProbs ? 9 : 1);
+    }
+    for (int s = 0; s < 8; ++s) {
+      mbar_init(k_full(s), 1);
+      mbar_init(k_empty(s), 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(t_full(s), 1);
+      mbar_init(t_empty(s), 4);
+    }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0;
+    *never = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_addr(const_cast<uint32_t*>(tmem_slot)), 2 * kSlotCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  bool failed = false;
+
+  if (warp == 0) {
+    // ---------------- producer: Q rows (+ row statistics) per item, K tiles ----------------
+    if (lane == 0) {
+      prefetch_tensormap(&mapQ);
+      prefetch_tensormap(&mapK);
+    }
+    uint32_t it_k = 0, item_cnt = 0;
+    uint32_t armed = 0, last_phase = 0;
+    bool q_armed = false;
+    uint32_t q_last = 0;
+    for (long long item = blockIdx.x; item < a.nitems; item += gridDim.x, ++item_cnt) {
+      const Item w = decode_item(item, a);
+      const int qb = item_cnt % a.qbufs;
+      const uint32_t qph = (item_cnt / a.qbufs) & 1u;
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait_bounded(q_empty(qb), qph ^ 1u, abort_flag);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { failed = true; break; }
+      if (PASS == kProbs) {
+        // the normalisation constants of the group's rows, next to the Q buffer they belong to
+        float2* dst = stats + qb * a.rows;
+        for (int r = lane; r < a.rows; r += 32) {
+          const long long rowg = ((long long)w.b * a.Hq + (long long)w.g * a.G + r / W) * W + r % W;
+          dst[r] = make_float2(-a.rowstat[2 * rowg] * kLog2e, a.rowstat[2 * rowg + 1]);
+        }
+        __syncwarp();
+      }
+      if (lane == 0) {
+        mbar_arrive_expect_tx(q_full(qb), (uint32_t)(a.rows * DH * 2));
+#pragma unroll
+        for (int p = 0; p < kPanels; ++p)
+          tma_load_4d(sbase + qb * L.q_bytes + p * L.q_panel, &mapQ, p * 64, 0, w.g * a.G, w.b, q_full(qb));
+        q_armed = true;
+        q_last = (uint32_t)qb | (qph << 1);
+        for (int t = w.t0; t < w.t1; ++t, ++it_k) {
+          const int s = it_k % a.kstages;
+          const uint32_t ph = (it_k / a.kstages) & 1u;
+          if (!mbar_wait_bounded(k_empty(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_arrive_expect_tx(k_full(s), (uint32_t)L.k_stage);
+          const uint32_t dst = sbase + L.k_off + s * L.k_stage;
+#pragma unroll
+          for (int p = 0; p < kPanels; ++p)
+            tma_load_4d(dst + p * (kKeyTile * 128), &mapK, p * 64, t * kKeyTile, w.g, w.b, k_full(s));
+          armed |= 1u << s;
+          last_phase = (last_phase & ~(1u << s)) | (ph << s);
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { failed = true; break; }
+    }
+    if (failed && lane == 0) {
+      if (q_armed) mbar_wait_bounded(q_full(q_last & 1u), q_last >> 1, never, 200000000ull);
+      for (int s = 0; s < a.kstages; ++s)
+        if (armed & (1u << s)) mbar_wait_bounded(k_full(s), (last_phase >> s) & 1u, never, 200000000ull);
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      uint32_t it_k = 0, item_cnt = 0, t = 0;
+      for (long long item = blockIdx.x; item < a.nitems && !failed; item += gridDim.x, ++item_cnt) {
+        const Item w = decode_item(item, a);
+        const int qb = item_cnt % a.qbufs;
+        const uint32_t q_addr = sbase + qb * L.q_bytes;
+        if (!mbar_wait_bounded(q_full(qb), (item_cnt / a.qbufs) & 1u, abort_flag)) { failed = true; break; }
+        for (int kt = w.t0; kt < w.t1 && !failed; ++kt, ++it_k) {
+          const int s = it_k % a.kstages;
+          if (!mbar_wait_bounded(k_full(s), (it_k / a.kstages) & 1u, abort_flag)) { failed = true; break; }
+          const uint32_t k_addr = sbase + L.k_off + s * L.k_stage;
+          for (int sub = 0; sub < nsub; ++sub, ++t) {
+            const uint32_t slot = t & 1u;
+            if (!mbar_wait_bounded(t_empty(slot), ((t >> 1) & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+            tc_fence_after();
+            uint32_t idesc, a_addr, b_addr, a_panel, b_panel;
+            if (PASS == kStats) {
+              // rows = query rows [sub*128, sub*128+128) of the group, columns = the 128 keys of the tile
+              idesc = idesc_bf16_f32(128, kKeyTile, 0);
+              a_addr = q_addr + sub * (128 * 128);
+              a_panel = L.q_panel;
+              b_addr = k_addr;
+              b_panel = kKeyTile * 128;
+            } else {
+              // rows = the 128 keys of the tile, columns = the window rows of this head group
+              const int h0 = sub * a.heads_per_group;
+              const int ncols = min(a.heads_per_group, a.G - h0) * W;
+              idesc = idesc_bf16_f32(128, ncols, 0);
+              a_addr = k_addr;
+              a_panel = kKeyTile * 128;
+              b_addr = q_addr + h0 * W * 128;
+              b_panel = L.q_panel;
+            }
+#pragma unroll
+            for (int kk = 0; kk < kKSteps; ++kk) {
+              const uint64_t ad = smem_desc_sw128(a_addr + (kk / 4) * a_panel + (kk % 4) * 32, 16, 1024);
+              const uint64_t bd = smem_desc_sw128(b_addr + (kk / 4) * b_panel + (kk % 4) * 32, 16, 1024);
+              umma_f16(tmem_base + slot * kSlotCols, ad, bd, idesc, kk > 0 ? 1u : 0u);
+            }
+            umma_commit(t_full(slot));
+          }
+          if (failed) break;
+          umma_commit(k_empty(s));
+        }
+        if (failed) break;
+        umma_commit(q_empty(qb));
+      }
+      umma_commit(drain_bar);
+      mbar_wait_bounded(drain_bar, 0, never, 500000000ull);
+    }
+  } else {
+    // ---------------- softmax warps: set = (warp - 2) / 4 takes the accumulators with t % 2 == set ----------------
+    const uint32_t set = (uint32_t)(warp - 2) >> 2;
+    const int quad = warp & 3;
+    const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + set * kSlotCols;
+    const int first_pos = a.n - W;  // sequence position of window row 0
+    uint32_t item_cnt = 0, t = 0, uses = 0;
+    for (long long item = blockIdx.x; item < a.nitems && !failed; item += gridDim.x, ++item_cnt) {
+      const Item w = decode_item(item, a);
+      const int qb = item_cnt % a.qbufs;
+      if (PASS == kProbs) {
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(q_full(qb), (item_cnt / a.qbufs) & 1u, abort_flag))) {
+          failed = true;
+          break;
+        }
+      }
+      const float2* st = stats + qb * a.rows;
+      float rm[kMaxRowBlocks], rl[kMaxRowBlocks];
+#pragma unroll
+      for (int rb = 0; rb < kMaxRowBlocks; ++rb) { rm[rb] = -INFINITY; rl[rb] = 0.f; }
+
+      for (int kt = w.t0; kt < w.t1 && !failed; ++kt) {
+        const int key0 = kt * kKeyTile;
+        const bool tail = key0 + kKeyTile - 1 > first_pos;  // some (key, row) pair of this tile is masked
+#pragma unroll 1
+        for (int sub = 0; sub < nsub; ++sub, ++t) {
+          if ((t & 1u) != set) continue;
+          if (!__all_sync(0xffffffffu, mbar_wait_bounded(t_full(set), uses & 1u, abort_flag))) { failed = true; break; }
+          ++uses;
+          tc_fence_after();
+          if (PASS == kStats) {
+            const int r = sub * 128 + quad * 32 + lane;           // query row of the group
+            const bool warp_live = sub * 128 + quad * 32 < a.rows;
+            float v[4][32];
+            if (warp_live) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) tmem_ld_32cols(lane_base + q * 32, v[q]);
+              tc_wait_ld();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(t_empty(set));
+            if (warp_live && r < a.rows) {
+              const int lim = min(first_pos + r % W, a.n - 1);    // last visible key of this row
+              float mx = -INFINITY;
+#pragma unroll
+              for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                  if (tail && key0 + q * 32 + e > lim) v[q][e] = -INFINITY;
+                  mx = fmaxf(mx, v[q][e]);
+                }
+              float m_old = -INFINITY, l_old = 0.f;
+#pragma unroll
+              for (int rb = 0; rb < kMaxRowBlocks; ++rb)
+                if (rb == sub) { m_old = rm[rb]; l_old = rl[rb]; }
+              const float m_new = fmaxf(m_old, mx);
+              if (m_new > -INFINITY) {
+                const float mc = m_new * a.c;
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                  s0 += ex2_approx(fmaf(v[0][e], a.c, -mc));
+                  s1 += ex2_approx(fmaf(v[1][e], a.c, -mc));
+                  s2 += ex2_approx(fmaf(v[2][e], a.c, -mc));
+                  s3 += ex2_approx(fmaf(v[3][e], a.c, -mc));
+                }
+                l_old = l_old * ex2_approx((m_old - m_new) * a.c) + ((s0 + s1) + (s2 + s3));
+                m_old = m_new;
+              }
+#pragma unroll
+              for (int rb = 0; rb < kMaxRowBlocks; ++rb)
+                if (rb == sub) { rm[rb] = m_old; rl[rb] = l_old; }
+            }
+          } else {
+            const int i = key0 + quad * 32 + lane;               // this thread's key
+            const int h0 = sub * a.heads_per_group;
+            const int nh = min(a.heads_per_group, a.G - h0);
+            for (int hq = 0; hq < nh; ++hq) {
+              float v[W / 16][16];
+#pragma unroll
+              for (int q = 0; q < W / 16; ++q) tmem_ld_16cols(lane_base + hq * W + q * 16, v[q]);
+              tc_wait_ld();
+              if (hq == nh - 1) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(t_empty(set));
+              }
+              const float2* sr = st + (h0 + hq) * W;
+              float acc = 0.f;
+#pragma unroll
+              for (int j = 0; j < W; ++j) {
+                const float2 c2 = sr[j];
+                float p = ex2_approx(fmaf(v[j / 16][j % 16], a.c, c2.x)) * c2.y;
+                if (tail && i > first_pos + j) p = 0.f;
+                acc += p;
+              }
+              if (i < a.n) a.abar[((long long)w.b * a.Hq + (long long)w.g * a.G + h0 + hq) * a.n + i] = acc;
+            }
+          }
+        }
+      }
+      if (PASS == kProbs && !failed) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(q_empty(qb));
+      }
+      if (PASS == kStats && !failed) {
+#pragma unroll
+        for (int rb = 0; rb < kMaxRowBlocks; ++rb) {
+          const int r = rb * 128 + quad * 32 + lane;
+          if (rb < a.row_blocks && r < a.rows) {
+            const long long rowg = ((long long)w.b * a.Hq + (long long)w.g * a.G + r / W) * W + r % W;
+            const long long o = rowg * a.part_stride + w.chunk * 2 + set;
+            a.part_m[o] = rm[rb] * a.scale;
+            a.part_l[o] = rl[rb];
+          }
+        }
+      }
+    }
+  }
+
+  if (failed) {
+    *abort_flag = 1;
+    atomicExch(a.status, (int)CKV_ETIMEOUT);
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 2 * kSlotCols);
+  }
+}
+
+template <int DH, int W, int PASS>
+cudaError_t run_pass(const CUtensorMap& mq, const CUtensorMap& mk, const AttnUmmaArgs& a, int grid,
+                     cudaStream_t st) {
+  const Layout<DH> L(a.rows, a.kstages, a.qbufs);
+  const int smem = L.total + 1024;
+  auto k = window_attn_umma_kernel<DH, W, PASS>;
+  cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  k<<<grid, kThreads, smem, st>>>(mq, mk, a);
+  return cudaGetLastError();
+}
+
+template <int DH, int W>
+cudaError_t run_both(const Dims& d, const CUtensorMap& mq, const CUtensorMap& mk, AttnUmmaArgs& a, int grid,
+                     float* attn, const ScoreWorkspace& ws, cudaStream_t st, int* launches) {
+  cudaError_t e = run_pass<DH, W, kStats>(mq, mk, a, grid, st);
+  if (e != cudaSuccess) return e;
+  e = launch_attn_combine(ws.part_m, ws.part_l, ws.rowstat, d.nb * d.Hq * d.w, a.part_stride, d.w, st);
+  if (e != cudaSuccess) return e;
+  e = run_pass<DH, W, kProbs>(mq, mk, a, grid, st);
+  if (e != cudaSuccess) return e;
+  e = launch_maxpool(ws.abar, attn, d.n, d.kp, d.nb * d.Hq, st);
+  *launches += 4;
+  return e;
+}
+
+}  // namespace
+
+cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K, float* attn,
+                                    const ScoreWorkspace& ws, int sm_count, int* status_word, cudaStream_t st,
+                                    int* launches) {
+  if (d.dtype != CKV_BF16 || tma_encode_fn() == nullptr) return cudaErrorNotSupported;
+  if (d.w != 16 && d.w != 32 && d.w != 64) return cudaErrorNotSupported;
+  const int rows = d.G * d.w;
+  if (rows > 128 * kMaxRowBlocks) return cudaErrorNotSupported;
+
+  AttnUmmaArgs a;
+  a.part_m = ws.part_m; a.part_l = ws.part_l; a.rowstat = ws.rowstat; a.abar = ws.abar; a.status = status_word;
+  a.Hq = d.Hq; a.Hkv = d.Hkv; a.G = d.G; a.n = d.n; a.nb = d.nb;
+  a.rows = rows;
+  a.row_blocks = (rows + 127) / 128;
+  a.heads_per_group = kSlotCols / d.w < d.G ? kSlotCols / d.w : d.G;
+  a.head_groups = (d.G + a.heads_per_group - 1) / a.heads_per_group;
+  a.ntiles = (d.n + kKeyTile - 1) / kKeyTile;
+  // enough work items to fill the machine a few times over, but at least 4 key tiles each so that the partial
+  // statistics (two per item) fit the workspace sized for one partial per 256 keys
+  const long long groups = (long long)d.nb * d.Hkv;
+  long long want_items = 4LL * sm_count;
+  int tpi = (int)((groups * a.ntiles + want_items - 1) / want_items);
+  if (tpi < 4) tpi = 4;
+  if (tpi > 64) tpi = 64;
+  a.tiles_per_item = tpi;
+  a.chunks_per_bg = (a.ntiles + tpi - 1) / tpi;
+  a.part_stride = 2 * a.chunks_per_bg;
+  if (a.part_stride > (d.n + kAttnChunk - 1) / kAttnChunk + 2) return cudaErrorNotSupported;  // workspace layout
+  a.nitems = groups * a.chunks_per_bg;
+  a.scale = d.scale;
+  a.c = d.scale * kLog2e;
+  // shared memory: Q rows, then as many K stages as fit (2..8)
+  const int q_bytes = ((rows * 128 * (d.dh / 64)) + 1023) / 1024 * 1024;
+  const int k_stage = kKeyTile * d.dh * 2;
+  const int budget = 225 * 1024 - 2 * rows * 8 - 1024;
+  a.qbufs = (budget - 2 * q_bytes) / k_stage >= 3 ? 2 : 1;
+  int ks = (budget - a.qbufs * q_bytes) / k_stage;
+  if (ks > 8) ks = 8;
+  if (ks < 2) return cudaErrorNotSupported;
+  a.kstages = ks;
+
+  CUtensorMap mq, mk;
+  const cuuint64_t qdims[4] = {(cuuint64_t)d.dh, (cuuint64_t)d.w, (cuuint64_t)d.Hq, (cuuint64_t)d.nb};
+  const long long qstr[3] = {d.qs[2], d.qs[1], d.qs[0]};
+  const cuuint32_t qbox[4] = {64, (cuuint32_t)d.w, (cuuint32_t)d.G, 1};
+  if (!make_bf16_map_4d(&mq, Qw, qdims, qstr, qbox)) return cudaErrorNotSupported;
+  const cuuint64_t kdims[4] = {(cuuint64_t)d.dh, (cuuint64_t)d.n, (cuuint64_t)d.Hkv, (cuuint64_t)d.nb};
+  const long long kstr[3] = {d.ks[2], d.ks[1], d.ks[0]};
+  const cuuint32_t kbox[4] = {64, kKeyTile, 1, 1};
+  if (!make_bf16_map_4d(&mk, K, kdims, kstr, kbox)) return cudaErrorNotSupported;
+
+  const int grid = (int)(a.nitems < sm_count ? a.nitems : sm_count);
+#define CKV_ATTN_CASE(DHV, WV) \
+  if (d.dh == DHV && d.w == WV) return run_both<DHV, WV>(d, mq, mk, a, grid, attn, ws, st, launches);
+  CKV_ATTN_CASE(128, 16) CKV_ATTN_CASE(128, 32) CKV_ATTN_CASE(128, 64)
+  CKV_ATTN_CASE(64, 16) CKV_ATTN_CASE(64, 32) CKV_ATTN_CASE(64, 64)
+#undef CKV_ATTN_CASE
+  return cudaErrorNotSupported;
+}
+
+}  // namespace ckv

@@ -39,15 +39,35 @@ SMALL = [
     dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=0.25),
     dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=1.0),
     dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=0.0),
+    # shapes the tensor-core kernels take (w in {16, 32, 64}), with ragged last tiles and short last work items
+    dict(dtype="bf16", n=700, w=32, kp=7, budget=90, dh=128, dm=384, Hq=8, Hkv=2),
+    dict(dtype="bf16", n=3000, w=64, kp=7, budget=250, dh=128, dm=640, Hq=10, Hkv=2),    # 320 query rows per group
+    dict(dtype="bf16", n=1000, w=16, kp=5, budget=77, dh=64, dm=192, Hq=4, Hkv=2),
+    dict(dtype="bf16", n=130, w=64, kp=3, budget=40, dh=128, dm=128, Hq=2, Hkv=2),
+    dict(dtype="bf16", n=5000, w=32, kp=7, budget_mode="adaptive", budget=2000, dh=128, dm=1024, Hq=16, Hkv=4),
 ]
+TENSOR_CORE_CASES = range(12, 17)
 
 
 @pytest.mark.parametrize("case", range(len(SMALL)))
 def test_small_and_edge_cases(case):
     wl = small_workload(cfg_id=100 + case, **SMALL[case])
-    Ls, outs, _ = _run(wl, layers=(0, 1))
+    Ls, outs, s = _run(wl, layers=(0, 1))
+    if case in TENSOR_CORE_CASES:
+        assert s.last_path == 3, "expected the tcgen05 kernels for window attention and projection norm"
     for L, out in zip(Ls, outs):
         pu.check_layer_against_oracle(L, wl, out)
+
+
+def test_forced_cuda_core_path_agrees_with_tensor_core_path():
+    from paper_2502_03805_b200 import binding as B
+    wl = small_workload(cfg_id=131, dtype="bf16", n=1300, w=32, kp=7, budget=200, dh=128, dm=512, Hq=8, Hkv=2)
+    Ls, tc, s1 = _run(wl)
+    _, cc, s2 = _run(wl, flags=B.CKV_FLAG_FORCE_SIMT)
+    assert s1.last_path == 3 and s2.last_path == 12
+    pu.assert_scores_close(tc[0]["attn"], cc[0]["attn"], "attn", rtol=1e-4)
+    pu.assert_scores_close(tc[0]["vnorm"], cc[0]["vnorm"], "vnorm", rtol=1e-4)
+    pu.check_layer_against_oracle(Ls[0], wl, cc[0])
 
 
 def test_separate_calls_equal_fused_call_and_are_deterministic():
@@ -130,14 +150,16 @@ def test_strided_kv_layout():
 
 def test_config1_full_parity():
     wl = config(1)
-    Ls, outs, _ = _run(wl)
+    Ls, outs, s = _run(wl)
+    assert s.last_path == 3
     rep = pu.check_layer_against_oracle(Ls[0], wl, outs[0])
     print("config1", rep)
 
 
 def test_config2_full_parity():
     wl = config(2)
-    Ls, outs, _ = _run(wl)
+    Ls, outs, s = _run(wl)
+    assert s.last_path == 3
     rep = pu.check_layer_against_oracle(Ls[0], wl, outs[0], full_output_check=True)
     print("config2", rep)
 
@@ -147,7 +169,8 @@ def test_config3_two_layers_adaptive_parity():
     wl = config(3)
     shares = [make_layer(wl.with_(n=64, dm=8), l).share_target for l in range(wl.layers)]
     layers = (int(np.argmin(shares)), int(np.argmax(shares)))
-    Ls, outs, _ = _run(wl, layers=layers)
+    Ls, outs, s = _run(wl, layers=layers)
+    assert s.last_path == 3
     for L, out in zip(Ls, outs):
         rep = pu.check_layer_against_oracle(L, wl, out)
         print("config3 layer", L.layer, rep)
@@ -160,7 +183,8 @@ def test_config4_one_layer_sampled(mode):
     wl = config(4)
     if mode == "adaptive":
         wl = wl.with_(budget_mode="adaptive", budget=8 * wl.budget)
-    Ls, outs, _ = _run(wl)
+    Ls, outs, s = _run(wl)
+    assert s.last_path == 3
     L, out = Ls[0], outs[0]
     P = oc.pooled_window_attention(L.Qw, L.K, wl.kp, wl.scale)
     pu.assert_scores_close(out["attn"], P, "attn")
