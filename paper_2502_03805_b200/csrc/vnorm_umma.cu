@@ -2,15 +2,20 @@
 // row of V W^O"; Theorem 3.3), bf16 inputs, float32 accumulation in tensor memory, and an epilogue that reduces every
 // output row to its L1 norm so the n x dm product never leaves the SM.
 //
-// Persistent kernel, one CTA per SM, 7 warps with fixed roles:
+// Persistent kernel, one CTA per SM, 11 warps with fixed roles:
 //   warp 0  B producer : TMA loads of W^O_h column chunks (kNC columns x dh), kStages deep
 //   warp 1  MMA issuer : tcgen05.mma 128 x kNC x 16, dh/16 per (chunk, token tile); owns the TMEM allocation
 //   warp 2  A producer : TMA loads of the work item's kTiles token tiles of V (128 tokens x dh each), resident for
 //                        the whole item
-//   warps 3-6 epilogue : tcgen05.ld of a finished 128 x kNC accumulator, |x| summed into one register per row
+//   warps 3-10 epilogue: two sets of four warps (one warp per 32-lane quarter of tensor memory); set s takes the
+//                        token tiles with (tile & 1) == s: tcgen05.ld of a finished 128 x kNC accumulator, |x| summed
+//                        into one register per row
 // A work item is (nb slice, query head, block of kTiles*128 tokens).  Each W^O chunk fetched from L2 is used by all
 // kTiles token tiles, which cuts the shared-memory fill per flop by kTiles; the kTiles accumulators (kTiles * kNC =
-// 512 columns, all of tensor memory) let the epilogue of one tile overlap the MMAs of the next three.
+// 512 columns, all of tensor memory) let the epilogue of one tile overlap the MMAs of the next.
+// Shape choice (measured): with 128 x 128 x 16 MMAs both operands stream from shared memory at 128 B/cycle, the
+// whole shared-memory bandwidth of the SM, and the tensor pipe idles half of the time (1150 TFLOP/s); 128 x 256 x 16
+// needs 96 B/cycle and reaches 1500 TFLOP/s.  Hence kNC = 256 with two token tiles and a two-deep W^O ring.
 // Operand layouts: V rows are K-major (dh contiguous); W^O_h is N-major (dm contiguous), consumed directly through an
 // MN-major shared-memory descriptor, so no transposed copy of W^O is ever made.  128-byte swizzle on both.
 // Every wait is bounded: when one runs out the kernel records CKV_ETIMEOUT in the status word, drains what it has in
@@ -26,10 +31,20 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kTiles = 4;       // token tiles (128 rows) per work item
-constexpr int kNC = 128;        // W^O columns per chunk = MMA N
-constexpr int kStages = 3;      // W^O chunk ring
-constexpr int kThreads = 7 * 32;
+#ifndef CKV_VN_TILES
+#define CKV_VN_TILES 2
+#endif
+#ifndef CKV_VN_NC
+#define CKV_VN_NC 256
+#endif
+#ifndef CKV_VN_STAGES
+#define CKV_VN_STAGES 2
+#endif
+constexpr int kTiles = CKV_VN_TILES;    // token tiles (128 rows) per work item
+constexpr int kNC = CKV_VN_NC;          // W^O columns per chunk = MMA N
+constexpr int kStages = CKV_VN_STAGES;  // W^O chunk ring
+static_assert(kTiles * kNC <= 512 && kNC % 128 == 0 && kNC <= 256, "accumulators must fit tensor memory");
+constexpr int kThreads = 11 * 32;
 constexpr int kTmemCols = kTiles * kNC;  // 512
 
 struct UmmaArgs {
@@ -138,9 +153,15 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
           if (!mbar_wait_bounded(b_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
           mbar_arrive_expect_tx(b_full(s), L::kBStage);
           const uint32_t dst = sbase + L::kBOff + s * L::kBStage;
+#ifdef CKV_VN_B_KMAJOR
+#pragma unroll
+          for (int p = 0; p < kPanels; ++p)
+            tma_load_4d(dst + p * (kNC * 128), &mapW, p * 64, j * kNC, w.h, bw, b_full(s));
+#else
 #pragma unroll
           for (int nbk = 0; nbk < kNC / 64; ++nbk)
             tma_load_4d(dst + nbk * (DH * 128), &mapW, j * kNC + nbk * 64, 0, w.h, bw, b_full(s));
+#endif
           armed |= 1u << s;
           last_phase = (last_phase & ~(1u << s)) | (ph << s);
         }
@@ -182,7 +203,11 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
+#ifdef CKV_VN_B_KMAJOR
+      constexpr uint32_t idesc = idesc_bf16_f32(128, kNC, 0);
+#else
       constexpr uint32_t idesc = idesc_bf16_f32(128, kNC, 1);
+#endif
       uint32_t it_b = 0, item_cnt = 0;
       uint32_t use[kTiles];
 #pragma unroll
@@ -209,7 +234,11 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
                 //    next 64-element panel = next 128-row block.  B: N-major, 64-column blocks DH*128 bytes apart
                 //    (leading offset), 8-row K groups 1024 bytes apart (stride offset); 16 K rows = 2048 bytes.
                 const uint64_t ad = smem_desc_sw128(a_addr + (kk / 4) * (128 * 128) + (kk % 4) * 32, 16, 1024);
+#ifdef CKV_VN_B_KMAJOR
+                const uint64_t bd = smem_desc_sw128(b_addr + (kk / 4) * (kNC * 128) + (kk % 4) * 32, 16, 1024);
+#else
                 const uint64_t bd = smem_desc_sw128(b_addr + kk * 2048, DH * 128, 1024);
+#endif
                 umma_f16(tmem_base + m * kNC, ad, bd, idesc, kk > 0 ? 1u : 0u);
               }
               umma_commit(t_full(m));
@@ -226,8 +255,9 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
       mbar_wait_bounded(drain_bar, 0, never, 500000000ull);
     }
   } else {
-    // ---------------- epilogue: warps 3..6 own TMEM lanes 32*(warp%4) .. +31 ----------------
+    // ---------------- epilogue: a warp owns TMEM lanes 32*(warp%4) .. +31 of the tiles of its set ----------------
     const int quad = warp & 3;
+    const int set = (warp - 3) >> 2;
     const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16);
     uint32_t use[kTiles];
 #pragma unroll
@@ -240,34 +270,39 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
       for (int j = 0; j < nchunks && !failed; ++j) {
 #pragma unroll
         for (int m = 0; m < kTiles; ++m) {
-          if (m >= w.tiles) continue;
+          if ((m & 1) != set || m >= w.tiles) continue;
           // the warp must stay converged for the .sync.aligned loads: all lanes succeed or all give up
           if (!__all_sync(0xffffffffu, mbar_wait_bounded(t_full(m), use[m] & 1u, abort_flag))) { failed = true; break; }
           ++use[m];
           tc_fence_after();
-          float v[4][32];
 #pragma unroll
-          for (int q = 0; q < kNC / 32; ++q) tmem_ld_32cols(lane_base + m * kNC + q * 32, v[q]);
-          tc_wait_ld();
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(t_empty(m));
-          float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+          for (int half = 0; half < kNC / 128; ++half) {
+            float v[4][32];
 #pragma unroll
-          for (int e = 0; e < 32; ++e) {
-            s0 += fabsf(v[0][e]);
-            s1 += fabsf(v[1][e]);
-            s2 += fabsf(v[2][e]);
-            s3 += fabsf(v[3][e]);
+            for (int q = 0; q < 4; ++q) tmem_ld_32cols(lane_base + m * kNC + half * 128 + q * 32, v[q]);
+            tc_wait_ld();
+            if (half == kNC / 128 - 1) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(t_empty(m));
+            }
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+              s0 += fabsf(v[0][e]);
+              s1 += fabsf(v[1][e]);
+              s2 += fabsf(v[2][e]);
+              s3 += fabsf(v[3][e]);
+            }
+            acc[m] += (s0 + s1) + (s2 + s3);
           }
-          acc[m] += (s0 + s1) + (s2 + s3);
         }
       }
       if (!failed) {
 #pragma unroll
         for (int m = 0; m < kTiles; ++m) {
           const int i = w.row0 + m * 128 + quad * 32 + lane;
-          if (m < w.tiles && i < a.n) a.vnorm[((long long)w.b * a.Hq + w.h) * a.n + i] = acc[m];
+          if ((m & 1) == set && m < w.tiles && i < a.n) a.vnorm[((long long)w.b * a.Hq + w.h) * a.n + i] = acc[m];
         }
       }
     }
@@ -316,9 +351,16 @@ cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, floa
   const cuuint32_t vbox[4] = {64, 128, 1, 1};
   if (!make_bf16_map_4d(&mv, V, vdims, vstr, vbox)) return cudaErrorNotSupported;
   const int nbw = d.wo_shared ? 1 : d.nb;
+#ifdef CKV_VN_B_KMAJOR
+  // experiment: WO given transposed, [nbw, Hq, dm, dh]
+  const cuuint64_t wdims[4] = {(cuuint64_t)d.dh, (cuuint64_t)d.dm, (cuuint64_t)d.Hq, (cuuint64_t)nbw};
+  const long long wstr[3] = {d.dh, (long long)d.dh * d.dm, (long long)d.Hq * d.dh * d.dm};
+  const cuuint32_t wbox[4] = {64, (cuuint32_t)kNC, 1, 1};
+#else
   const cuuint64_t wdims[4] = {(cuuint64_t)d.dm, (cuuint64_t)d.dh, (cuuint64_t)d.Hq, (cuuint64_t)nbw};
   const long long wstr[3] = {d.dm, (long long)d.dh * d.dm, (long long)d.Hq * d.dh * d.dm};
   const cuuint32_t wbox[4] = {64, (cuuint32_t)d.dh, 1, 1};
+#endif
   if (!make_bf16_map_4d(&mw, WO, wdims, wstr, wbox)) return cudaErrorNotSupported;
   UmmaArgs a;
   a.vnorm = vnorm; a.status = status_word;
