@@ -275,39 +275,31 @@ def main():
 
 
 def run_e2e(args, wl, host, local, world):
-    """Same metric with every step's inputs starting in pinned host memory and its results ending there.
-    Layers are streamed one at a time: copy-in, compress and copy-out of neighbouring layers overlap on two
-    streams with double-buffered device staging."""
+    """Same metric through criticalkv_compress_host: every step's inputs start in pinned host memory and its results
+    (idx, offsets, compacted K and V) end there; the library streams the layers through two device staging buffers."""
     import torch
     import torch.distributed as dist
-    from paper_2502_03805_b200 import session_for
+    from paper_2502_03805_b200 import binding as B
+    from paper_2502_03805_b200.dist_util import max_over_ranks, whole_job_throughput
     dev = torch.device("cuda", local)
     nb = wl.layers
     tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
-    sess = [session_for(wl, nb=1, device=local, want_stage=False) for _ in range(2)]
-    stage_in = [{k: torch.empty_like(v[0:1], device=dev) for k, v in host.items()} for _ in range(2)]
+    desc = B.make_desc(nb=nb, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp, dtype=wl.dtype,
+                       budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps)
+    handle = B.criticalkv_create(local)
+    staging = torch.empty(B.criticalkv_host_staging_bytes(desc), dtype=torch.uint8, device=dev)
     out_host = {"idx": torch.empty((nb, wl.btot), dtype=torch.int32).pin_memory(),
                 "offsets": torch.empty((nb, wl.Hkv + 1), dtype=torch.int32).pin_memory(),
                 "K_out": torch.empty((nb, wl.btot, wl.dh), dtype=tdt).pin_memory(),
                 "V_out": torch.empty((nb, wl.btot, wl.dh), dtype=tdt).pin_memory()}
-    streams = [torch.cuda.Stream(device=dev) for _ in range(2)]
-    h2d = sum(v[0:1].numel() * v.element_size() for v in host.values()) * nb
-    d2h = sum(v[0:1].numel() * v.element_size() for v in out_host.values()) * nb
+    h2d = sum(v.numel() * v.element_size() for v in host.values())
+    d2h = sum(v.numel() * v.element_size() for v in out_host.values())
+    stream = torch.cuda.current_stream()
 
     def step():
-        for l in range(nb):
-            p = l & 1
-            st, ss, si = streams[p], sess[p], stage_in[p]
-            with torch.cuda.stream(st):
-                for k in host:
-                    si[k].copy_(host[k][l:l + 1], non_blocking=True)
-                ss.compress(si["Qw_store"], si["K_store"], si["V_store"], si["WO_store"], stream=st)
-                out_host["idx"][l:l + 1].copy_(ss.idx, non_blocking=True)
-                out_host["offsets"][l:l + 1].copy_(ss.offsets, non_blocking=True)
-                out_host["K_out"][l:l + 1].copy_(ss.K_out, non_blocking=True)
-                out_host["V_out"][l:l + 1].copy_(ss.V_out, non_blocking=True)
-        for st in streams:
-            st.synchronize()
+        B.criticalkv_compress_host(handle, desc, host["Qw_store"], host["K_store"], host["V_store"], host["WO_store"],
+                                   None, out_host["idx"], out_host["offsets"], out_host["K_out"], out_host["V_out"],
+                                   staging, stream=stream)
 
     def barrier():
         if world > 1:
@@ -322,14 +314,14 @@ def run_e2e(args, wl, host, local, world):
     for _ in range(steps):
         step()
     barrier()
-    dt = time.perf_counter() - t0
-    from paper_2502_03805_b200.dist_util import max_over_ranks, whole_job_throughput
-    dt = max_over_ranks(dt, dev)
+    dt = max_over_ranks(time.perf_counter() - t0, dev)
+    assert B.criticalkv_device_status(handle) == 0
+    B.criticalkv_destroy(handle)
     value = whole_job_throughput(nb * wl.Hkv * wl.n * steps, world, dt)
     return {"value": value, "unit": UNIT, "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
             "ms_per_step": 1e3 * dt / steps, "steps": steps,
-            "how": "per layer: pinned host -> device copies of Qw, K, V, W_O, criticalkv_compress, device -> pinned "
-                   "host copies of idx, offsets, K_out, V_out; two streams, double-buffered"}
+            "how": "criticalkv_compress_host: pinned host Qw, K, V, W_O in; idx, offsets, K_out, V_out back to pinned "
+                   "host; layers streamed through two device staging buffers on two streams"}
 
 
 if __name__ == "__main__":

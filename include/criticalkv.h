@@ -15,7 +15,7 @@
  *     buffers, including the workspace; the library allocates device memory only in criticalkv_create (one status
  *     word).
  *   - Calls only enqueue work on the given CUDA stream (a cudaStream_t passed as void*, NULL = legacy default stream)
- *     and return; they never synchronise, except criticalkv_device_status.
+ *     and return; they never synchronise, except criticalkv_device_status and criticalkv_compress_host.
  *   - Return value: a criticalkv_status.  Argument errors are found on the host before any launch.  A device-side
  *     anomaly (a bounded wait that ran out) sets the handle's device status word; kernels still terminate.
  *   - Identical inputs give bit-identical outputs (no order-dependent floating-point atomics).
@@ -156,6 +156,30 @@ CKV_API int criticalkv_compress(criticalkv_handle h, const criticalkv_desc* d, c
                                 const void* V, const void* WO, const int32_t* budgets_in, float* attn, float* vnorm,
                                 int32_t* idx, int32_t* offsets, uint8_t* stage, void* K_out, void* V_out, void* ws,
                                 size_t ws_bytes, void* stream);
+
+/*
+ * The whole path for callers whose tensors live in HOST memory (pinned memory recommended): Qw, K, V, WO,
+ * budgets_in (given budgets only) are host arrays in the dense layouts above, idx [nb,Btot], offsets [nb,Hkv+1],
+ * K_out, V_out [nb,Btot,dh] are host arrays that receive the result.  The nb slices are streamed one at a time
+ * through two device staging buffers on two internal streams, so that the upload of slice b+1, the kernels of slice b
+ * and the download of slice b-1 overlap.  `staging` is DEVICE memory of at least criticalkv_host_staging_bytes(d),
+ * 256-byte aligned, owned by the caller; the call allocates no device memory (its first use on a handle creates two
+ * streams and three events).  Work starts after everything already queued on `stream`; unlike the other calls this
+ * one returns only when the results are in host memory.  Element strides in the descriptor must be 0 (dense).
+ */
+CKV_API int criticalkv_host_staging_bytes(const criticalkv_desc* d, size_t* bytes);
+CKV_API int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K,
+                                     const void* V, const void* WO, const int32_t* budgets_in, int32_t* idx,
+                                     int32_t* offsets, void* K_out, void* V_out, void* staging,
+                                     size_t staging_bytes, void* stream);
+
+/*
+ * Self-test of the bounded device-side wait every tensor-core kernel uses: launches one CTA that waits, for at most
+ * limit_ns nanoseconds, on a barrier nothing will ever signal.  The kernel must give up, write 0 to *observed_device
+ * (a device int; 1 would mean the wait claimed success), set the status word to CKV_ETIMEOUT and end normally.
+ */
+CKV_API int criticalkv_selftest_bounded_wait(criticalkv_handle h, uint64_t limit_ns, int* observed_device,
+                                             void* stream);
 
 /* Reads the device status word (synchronises `stream` first), clears it, and returns it in *out. */
 CKV_API int criticalkv_device_status(criticalkv_handle h, void* stream, int* out);

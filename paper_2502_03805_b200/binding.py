@@ -20,7 +20,8 @@ CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT = 1, 2
 CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",
-           "criticalkv_select", "criticalkv_select_static", "criticalkv_compact", "criticalkv_compress", "criticalkv_device_status",
+           "criticalkv_select", "criticalkv_select_static", "criticalkv_compact", "criticalkv_compress",
+           "criticalkv_host_staging_bytes", "criticalkv_compress_host", "criticalkv_selftest_bounded_wait", "criticalkv_device_status",
            "criticalkv_status_string", "criticalkv_last_cuda_error", "criticalkv_last_path",
            "criticalkv_launch_count")
 
@@ -63,6 +64,9 @@ def load():
     lib.criticalkv_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
     lib.criticalkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
     lib.criticalkv_compress.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.criticalkv_host_staging_bytes.argtypes = [dp, C.POINTER(sz)]
+    lib.criticalkv_compress_host.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.criticalkv_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp, vp]
     lib.criticalkv_device_status.argtypes = [vp, vp, C.POINTER(i32)]
     lib.criticalkv_status_string.argtypes = [i32]
     lib.criticalkv_status_string.restype = C.c_char_p
@@ -181,6 +185,28 @@ def criticalkv_compress(handle, desc, Qw, K, V, WO, budgets_in, attn, vnorm, idx
                                     _ptr(attn), _ptr(vnorm), _ptr(idx), _ptr(offsets), _ptr(stage), _ptr(K_out),
                                     _ptr(V_out), _ptr(ws), _nbytes(ws, ws_bytes), _stream(stream))
     return _check(handle, rc, "criticalkv_compress", check)
+
+
+def criticalkv_host_staging_bytes(desc):
+    out = C.c_size_t()
+    rc = load().criticalkv_host_staging_bytes(C.byref(desc), C.byref(out))
+    if rc != CKV_OK:
+        raise CriticalKVError(rc, "criticalkv_host_staging_bytes")
+    return out.value
+
+
+def criticalkv_compress_host(handle, desc, Qw, K, V, WO, budgets_in, idx, offsets, K_out, V_out, staging,
+                             staging_bytes=None, stream=None, check=True):
+    """Host tensors in (Qw, K, V, WO[, budgets_in]) and out (idx, offsets, K_out, V_out); `staging` is device memory."""
+    rc = load().criticalkv_compress_host(handle, C.byref(desc), _ptr(Qw), _ptr(K), _ptr(V), _ptr(WO),
+                                         _ptr(budgets_in), _ptr(idx), _ptr(offsets), _ptr(K_out), _ptr(V_out),
+                                         _ptr(staging), _nbytes(staging, staging_bytes), _stream(stream))
+    return _check(handle, rc, "criticalkv_compress_host", check)
+
+
+def criticalkv_selftest_bounded_wait(handle, limit_ns, observed, stream=None, check=True):
+    rc = load().criticalkv_selftest_bounded_wait(handle, int(limit_ns), _ptr(observed), _stream(stream))
+    return _check(handle, rc, "criticalkv_selftest_bounded_wait", check)
 
 
 def criticalkv_device_status(handle, stream=None):

@@ -17,6 +17,10 @@ struct criticalkv_handle_s {
   int last_path;
   long long launches;
   char cuda_error[256];
+  // host-staged path: two copy/compute streams and the events that tie them to the caller's stream
+  bool host_ready;
+  cudaStream_t host_stream[2];
+  cudaEvent_t host_event[3];
 };
 
 namespace {
@@ -161,6 +165,10 @@ int criticalkv_create(criticalkv_handle* out, int device) {
 int criticalkv_destroy(criticalkv_handle h) {
   if (!h) return CKV_EINVAL;
   DeviceGuard guard(h->device);
+  if (h->host_ready) {
+    for (int i = 0; i < 2; ++i) cudaStreamDestroy(h->host_stream[i]);
+    for (int i = 0; i < 3; ++i) cudaEventDestroy(h->host_event[i]);
+  }
   if (h->status_word) cudaFree(h->status_word);
   delete h;
   return CKV_OK;
@@ -290,6 +298,157 @@ int criticalkv_compress(criticalkv_handle h, const criticalkv_desc* d, const voi
   rc = criticalkv_select(h, d, attn, vnorm, budgets_in, idx, offsets, stage, ws, ws_bytes, stream);
   if (rc != CKV_OK) return rc;
   return criticalkv_compact(h, d, K, V, idx, offsets, K_out, V_out, stream);
+}
+
+// ---- host-staged compression ------------------------------------------------------------------------------------
+}  // extern "C"
+namespace {
+struct HostStaging {   // byte offsets inside one of the two device staging buffers
+  size_t Qw, K, V, WO, attn, vnorm, budgets, idx, offsets, K_out, V_out, ws, ws_bytes, total;
+  size_t nQw, nK, nV, nWO, nidx, noffsets, nout;   // bytes per nb slice
+};
+HostStaging host_staging_layout(const Dims& one) {
+  HostStaging L;
+  const size_t es = one.dtype == CKV_F32 ? 4 : 2;
+  L.nQw = (size_t)one.Hq * one.w * one.dh * es;
+  L.nK = L.nV = (size_t)one.Hkv * one.n * one.dh * es;
+  L.nWO = (size_t)one.Hq * one.dh * one.dm * es;
+  L.nidx = (size_t)one.btot * sizeof(int32_t);
+  L.noffsets = (size_t)(one.Hkv + 1) * sizeof(int32_t);
+  L.nout = (size_t)one.btot * one.dh * es;
+  const size_t nscore = (size_t)one.Hq * one.n * sizeof(float);
+  const size_t sb = score_layout(one).total, tb = select_layout(one).total;
+  L.ws_bytes = sb > tb ? sb : tb;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + (bytes ? bytes : 16), 256); return o; };
+  L.Qw = take(L.nQw); L.K = take(L.nK); L.V = take(L.nV); L.WO = take(L.nWO);
+  L.attn = take(nscore); L.vnorm = take(nscore);
+  L.budgets = take((size_t)one.Hkv * sizeof(int32_t));
+  L.idx = take(L.nidx); L.offsets = take(L.noffsets); L.K_out = take(L.nout); L.V_out = take(L.nout);
+  L.ws = take(L.ws_bytes);
+  L.total = off;
+  return L;
+}
+// Descriptor of a single dense nb slice of the caller's problem.
+criticalkv_desc single_slice_desc(const criticalkv_desc& d) {
+  criticalkv_desc o = d;
+  o.nb = 1;
+  for (int i = 0; i < 3; ++i) o.q_stride[i] = o.k_stride[i] = o.v_stride[i] = 0;
+  o.flags &= ~(uint32_t)CKV_FLAG_WO_SHARED;
+  return o;
+}
+}  // namespace
+extern "C" {
+
+int criticalkv_host_staging_bytes(const criticalkv_desc* d, size_t* bytes) {
+  if (!d || !bytes) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  criticalkv_desc one = single_slice_desc(*d);
+  Dims d1;
+  if ((rc = resolve(&one, &d1)) != CKV_OK) return rc;
+  *bytes = 2 * host_staging_layout(d1).total;
+  return CKV_OK;
+}
+
+int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K,
+                             const void* V, const void* WO, const int32_t* budgets_in, int32_t* idx,
+                             int32_t* offsets, void* K_out, void* V_out, void* staging, size_t staging_bytes,
+                             void* stream) {
+  if (!h || !d) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (!Qw || !K || !V || !WO || !idx || !offsets || !K_out || !V_out || !staging) return CKV_EINVAL;
+  if (dd.budget_mode == CKV_BUDGET_GIVEN && !budgets_in) return CKV_EINVAL;
+  for (int i = 0; i < 3; ++i)
+    if (d->q_stride[i] || d->k_stride[i] || d->v_stride[i]) return CKV_ENOTSUP;  // host arrays must be dense
+  if (reinterpret_cast<uintptr_t>(staging) & 255u) return CKV_EALIGN;
+  criticalkv_desc one = single_slice_desc(*d);
+  Dims d1;
+  if ((rc = resolve(&one, &d1)) != CKV_OK) return rc;
+  const HostStaging L = host_staging_layout(d1);
+  if (staging_bytes < 2 * L.total) return CKV_EWORKSPACE;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  cudaError_t e = cudaSuccess;
+  if (!h->host_ready) {
+    for (int i = 0; i < 2 && e == cudaSuccess; ++i)
+      e = cudaStreamCreateWithFlags(&h->host_stream[i], cudaStreamNonBlocking);
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i)
+      e = cudaEventCreateWithFlags(&h->host_event[i], cudaEventDisableTiming);
+    if (e != cudaSuccess) return record_cuda(h, e);
+    h->host_ready = true;
+  }
+  cudaStream_t user = (cudaStream_t)stream;
+  // the staging streams start after whatever the caller has queued on its stream
+  if ((e = cudaEventRecord(h->host_event[2], user)) != cudaSuccess) return record_cuda(h, e);
+  for (int i = 0; i < 2; ++i)
+    if ((e = cudaStreamWaitEvent(h->host_stream[i], h->host_event[2], 0)) != cudaSuccess) return record_cuda(h, e);
+
+  const bool wo_shared = dd.wo_shared != 0;
+  const char* hq = (const char*)Qw; const char* hk = (const char*)K; const char* hv = (const char*)V;
+  const char* hw = (const char*)WO;
+  for (int b = 0; b < dd.nb && rc == CKV_OK; ++b) {
+    const int p = b & 1;
+    cudaStream_t st = h->host_stream[p];
+    char* base = (char*)staging + (size_t)p * L.total;
+    // a shared W^O is uploaded once per staging buffer (slices 0 and 1)
+    const bool copy_wo = !wo_shared || b < 2;
+    if ((e = cudaMemcpyAsync(base + L.Qw, hq + (size_t)b * L.nQw, L.nQw, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(base + L.K, hk + (size_t)b * L.nK, L.nK, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(base + L.V, hv + (size_t)b * L.nV, L.nV, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
+        (copy_wo && (e = cudaMemcpyAsync(base + L.WO, hw + (wo_shared ? 0 : (size_t)b * L.nWO), L.nWO,
+                                         cudaMemcpyHostToDevice, st)) != cudaSuccess))
+      return record_cuda(h, e);
+    const int32_t* bud = nullptr;
+    if (dd.budget_mode == CKV_BUDGET_GIVEN) {
+      if ((e = cudaMemcpyAsync(base + L.budgets, budgets_in + (size_t)b * dd.Hkv, (size_t)dd.Hkv * sizeof(int32_t),
+                               cudaMemcpyHostToDevice, st)) != cudaSuccess)
+        return record_cuda(h, e);
+      bud = (const int32_t*)(base + L.budgets);
+    }
+    rc = criticalkv_score(h, &one, base + L.Qw, base + L.K, base + L.V, base + L.WO, (float*)(base + L.attn),
+                          (float*)(base + L.vnorm), base + L.ws, L.ws_bytes, st);
+    if (rc != CKV_OK) break;
+    rc = criticalkv_select(h, &one, (const float*)(base + L.attn), (const float*)(base + L.vnorm), bud,
+                           (int32_t*)(base + L.idx), (int32_t*)(base + L.offsets), nullptr, base + L.ws,
+                           L.ws_bytes, st);
+    if (rc != CKV_OK) break;
+    rc = criticalkv_compact(h, &one, base + L.K, base + L.V, (const int32_t*)(base + L.idx),
+                            (const int32_t*)(base + L.offsets), base + L.K_out, base + L.V_out, st);
+    if (rc != CKV_OK) break;
+    if ((L.nidx && (e = cudaMemcpyAsync((char*)idx + (size_t)b * L.nidx, base + L.idx, L.nidx,
+                                        cudaMemcpyDeviceToHost, st)) != cudaSuccess) ||
+        (e = cudaMemcpyAsync((char*)offsets + (size_t)b * L.noffsets, base + L.offsets, L.noffsets,
+                             cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+        (L.nout && ((e = cudaMemcpyAsync((char*)K_out + (size_t)b * L.nout, base + L.K_out, L.nout,
+                                         cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
+                    (e = cudaMemcpyAsync((char*)V_out + (size_t)b * L.nout, base + L.V_out, L.nout,
+                                         cudaMemcpyDeviceToHost, st)) != cudaSuccess)))
+      return record_cuda(h, e);
+  }
+  // join: the caller's stream continues after both staging streams, and the call returns with the results on the host
+  for (int i = 0; i < 2; ++i) {
+    cudaError_t e2 = cudaEventRecord(h->host_event[i], h->host_stream[i]);
+    if (e2 == cudaSuccess) e2 = cudaStreamWaitEvent(user, h->host_event[i], 0);
+    if (e == cudaSuccess) e = e2;
+  }
+  cudaError_t e3 = cudaStreamSynchronize(user);
+  if (e == cudaSuccess) e = e3;
+  if (rc != CKV_OK) return rc;
+  return record_cuda(h, e);
+}
+
+int criticalkv_selftest_bounded_wait(criticalkv_handle h, uint64_t limit_ns, int* observed_device, void* stream) {
+  if (!h || !observed_device) return CKV_EINVAL;
+  if (h->cc_major < 9) return CKV_ENOTSUP;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  cudaError_t e = ckv::launch_bounded_wait_selftest(h->status_word, limit_ns, observed_device, (cudaStream_t)stream);
+  h->launches += 1;
+  return record_cuda(h, e);
 }
 
 int criticalkv_device_status(criticalkv_handle h, void* stream, int* out) {

@@ -52,6 +52,8 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
 // the caller then uses the CUDA-core kernel.
 cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, float* vnorm, int sm_count,
                               int* status_word, cudaStream_t st, int* launches);
+cudaError_t launch_bounded_wait_selftest(int* status_word, unsigned long long limit_ns, int* observed,
+                                         cudaStream_t st);
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word);

@@ -148,6 +148,72 @@ def test_strided_kv_layout():
     pu.check_layer_against_oracle(L, wl, out)
 
 
+@pytest.mark.parametrize("mode,budget,shared", [("uniform", 90, False), ("adaptive", 400, True), ("given", 500, False)])
+def test_host_staged_compress_equals_device_compress(mode, budget, shared):
+    # criticalkv_compress_host with host arrays must give exactly what criticalkv_compress gives on device arrays
+    from paper_2502_03805_b200 import binding as B
+    from gpu_util import run_layers
+    wl = small_workload(cfg_id=151, dtype="bf16", n=900, w=32, kp=7, budget_mode=mode, budget=budget, dh=128,
+                        dm=256, Hq=8, Hkv=2)
+    nb = 3
+    Ls = [make_layer(wl, l) for l in range(nb)]
+    if shared:
+        for L in Ls[1:]:
+            L.WO_store, L.WO = Ls[0].WO_store, Ls[0].WO
+    budgets = np.array([[100, 400], [0, 250], [300, 200]], dtype=np.int32) if mode == "given" else None
+    flags = B.CKV_FLAG_WO_SHARED if shared else 0
+    desc = B.make_desc(nb=nb, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp, dtype="bf16",
+                       budget_mode=mode, budget=budget, flags=flags)
+    btot = budget * wl.Hkv if mode == "uniform" else budget
+
+    def pin(name, first_only=False):
+        arr = np.stack([getattr(L, name) for L in (Ls[:1] if first_only else Ls)])
+        return torch.from_numpy(arr).view(torch.bfloat16).pin_memory()
+    hQ, hK, hV, hW = pin("Qw_store"), pin("K_store"), pin("V_store"), pin("WO_store", first_only=shared)
+    hb = torch.from_numpy(budgets).pin_memory() if budgets is not None else None
+    idx = torch.full((nb, btot), -1, dtype=torch.int32).pin_memory()
+    off = torch.zeros((nb, wl.Hkv + 1), dtype=torch.int32).pin_memory()
+    Ko = torch.zeros((nb, btot, wl.dh), dtype=torch.bfloat16).pin_memory()
+    Vo = torch.zeros_like(Ko).pin_memory()
+    h = B.criticalkv_create(0)
+    staging = torch.empty(B.criticalkv_host_staging_bytes(desc), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        B.criticalkv_compress_host(h, desc, hQ, hK, hV, hW, hb, idx, off, Ko, Vo, staging)
+    assert B.criticalkv_device_status(h) == 0
+    B.criticalkv_destroy(h)
+    # device path, one slice at a time
+    for b in range(nb):
+        wl_b = wl if mode != "given" else wl
+        from paper_2502_03805_b200 import session_for, to_device, to_host
+        s = session_for(wl_b, nb=1)
+        dQ, dK, dV, dW = (to_device(getattr(Ls[b], k)[None], "bf16") for k in ("Qw_store", "K_store", "V_store", "WO_store"))
+        bi = torch.from_numpy(budgets[b:b + 1]).cuda() if budgets is not None else None
+        s.compress(dQ, dK, dV, dW, budgets_in=bi)
+        torch.cuda.synchronize()
+        tot = int(s.offsets[0, -1])
+        np.testing.assert_array_equal(off[b].numpy(), to_host(s.offsets[0]))
+        np.testing.assert_array_equal(idx[b, :tot].numpy(), to_host(s.idx[0])[:tot])
+        np.testing.assert_array_equal(to_host(Ko[b])[:tot], to_host(s.K_out[0])[:tot])
+        np.testing.assert_array_equal(to_host(Vo[b])[:tot], to_host(s.V_out[0])[:tot])
+
+
+def test_bounded_wait_times_out_and_reports_status():
+    # a wait on a barrier nothing signals must end by itself, set CKV_ETIMEOUT, and leave the context usable
+    import time
+    from paper_2502_03805_b200 import binding as B
+    h = B.criticalkv_create(0)
+    observed = torch.full((1,), 7, dtype=torch.int32, device="cuda")
+    t0 = time.perf_counter()
+    B.criticalkv_selftest_bounded_wait(h, 2_000_000, observed)          # 2 ms
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0
+    assert int(observed.item()) == 0
+    assert B.criticalkv_device_status(h) == B.CKV_ETIMEOUT
+    assert B.criticalkv_device_status(h) == 0                            # reading clears it
+    assert float((torch.ones(4, device="cuda") * 2).sum().item()) == 8.0  # the context still works
+    B.criticalkv_destroy(h)
+
+
 def test_config1_full_parity():
     wl = config(1)
     Ls, outs, s = _run(wl)
