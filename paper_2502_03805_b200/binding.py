@@ -9,7 +9,9 @@ from __future__ import annotations
 import ctypes as C
 import os
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcriticalkv.so")
+# CRITICALKV_LIB may point at another build of the same library (e.g. one compiled with different tile shapes)
+_LIB_PATH = os.environ.get("CRITICALKV_LIB") or os.path.join(os.path.dirname(os.path.abspath(__file__)),
+                                                             "libcriticalkv.so")
 _lib = None
 
 CKV_OK, CKV_EINVAL, CKV_ENOTSUP, CKV_EALIGN, CKV_EWORKSPACE, CKV_ECUDA, CKV_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6

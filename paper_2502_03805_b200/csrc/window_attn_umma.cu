@@ -15,6 +15,8 @@
 // Persistent kernel, one CTA per SM: warp 0 streams K tiles (and the group's Q rows, once per work item) with TMA,
 // warp 1 issues the MMAs, warps 2-9 are two sets of four softmax warps that take alternating accumulators (two
 // 256-column TMEM slots), so that the exponentials of one tile overlap the MMAs and TMEM loads of the next.
+// The per-element work is one fma and one exp (plus a max in sweep 1): the normaliser 1 / (w * sum) enters sweep 2
+// as log2 in the exponent's bias, and every reduction runs as four independent chains.
 // All waits are bounded (status word CKV_ETIMEOUT, tensor memory freed, normal return).
 #include <cuda_bf16.h>
 #include <math.h>
@@ -29,7 +31,9 @@ namespace {
 using namespace ptx;
 
 constexpr int kKeyTile = 128;
-constexpr int kThreads = 10 * 32;
+// softmax warps per (accumulator, TMEM lane quarter); 2 (columns split between two warps) measured no faster
+constexpr int kHalves = 1;
+constexpr int kThreads = (2 + 8 * kHalves) * 32;
 constexpr int kSlotCols = 256;
 constexpr int kMaxRowBlocks = 3;  // G*w <= 384
 constexpr float kLog2e = 1.4426950408889634f;
@@ -112,7 +116,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + L.bar_off + 25 * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
   volatile uint32_t* never = tmem_slot + 2;
-  float2* stats = reinterpret_cast<float2*>(smem + L.stats_off);  // [2][rows]: (-max * log2e, 1 / (w * sum))
+  float* stats = reinterpret_cast<float*>(smem + L.stats_off);  // [2][rows]: -max * log2e + log2(1 / (w * sum))
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   constexpr int kKSteps = DH / 16;
@@ -124,7 +128,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       mbar_init(q_full(s), 1);
       // a Q buffer is free again when the MMAs of its item have retired and, in the second sweep, when all eight
       // softmax warps are done with the item's statistics
-      mbar_init(q_empty(s), PASS == kProbs ? 9 : 1);
+      mbar_init(q_empty(s), PASS == kProbs ? 1 + 8 * kHalves : 1);
     }
     for (int s = 0; s < 8; ++s) {
       mbar_init(k_full(s), 1);
@@ -132,7 +136,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(t_full(s), 1);
-      mbar_init(t_empty(s), 4);
+      mbar_init(t_empty(s), 4 * kHalves);
     }
     mbar_init(drain_bar, 1);
     *abort_flag = 0;
@@ -170,10 +174,10 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       if (!ok) { failed = true; break; }
       if (PASS == kProbs) {
         // the normalisation constants of the group's rows, next to the Q buffer they belong to
-        float2* dst = stats + qb * a.rows;
+        float* dst = stats + qb * a.rows;
         for (int r = lane; r < a.rows; r += 32) {
           const long long rowg = ((long long)w.b * a.Hq + (long long)w.g * a.G + r / W) * W + r % W;
-          dst[r] = make_float2(-a.rowstat[2 * rowg] * kLog2e, a.rowstat[2 * rowg + 1]);
+          dst[r] = fmaf(-a.rowstat[2 * rowg], kLog2e, log2f(a.rowstat[2 * rowg + 1]));
         }
         __syncwarp();
       }
@@ -258,8 +262,13 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       mbar_wait_bounded(drain_bar, 0, never, 500000000ull);
     }
   } else {
-    // ---------------- softmax warps: set = (warp - 2) / 4 takes the accumulators with t % 2 == set ----------------
-    const uint32_t set = (uint32_t)(warp - 2) >> 2;
+    // ---------------- softmax warps ----------------
+    // warp e = warp - 2: TMEM lane quarter = warp % 4 (fixed by the hardware), accumulator slot ("set") = (e / 4) % 2,
+    // column half = e / 8.  A set takes the accumulators with t % 2 == set; its kHalves warps per lane quarter split
+    // the columns (sweep 1: keys, sweep 2: heads) between them.
+    const int e_id = warp - 2;
+    const uint32_t set = (uint32_t)(e_id >> 2) & 1u;
+    const int half = e_id >> 3;
     const int quad = warp & 3;
     const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + set * kSlotCols;
     const int first_pos = a.n - W;  // sequence position of window row 0
@@ -273,7 +282,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
           break;
         }
       }
-      const float2* st = stats + qb * a.rows;
+      const float* st = stats + qb * a.rows;
       float rm[kMaxRowBlocks], rl[kMaxRowBlocks];
 #pragma unroll
       for (int rb = 0; rb < kMaxRowBlocks; ++rb) { rm[rb] = -INFINITY; rl[rb] = 0.f; }
@@ -288,27 +297,39 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
           ++uses;
           tc_fence_after();
           if (PASS == kStats) {
+            constexpr int CW = kKeyTile / kHalves;                // key columns per warp
             const int r = sub * 128 + quad * 32 + lane;           // query row of the group
             const bool warp_live = sub * 128 + quad * 32 < a.rows;
-            float v[4][32];
+            const int c0 = half * CW;
+            float v[CW / 32][32];
             if (warp_live) {
 #pragma unroll
-              for (int q = 0; q < 4; ++q) tmem_ld_32cols(lane_base + q * 32, v[q]);
+              for (int q = 0; q < CW / 32; ++q) tmem_ld_32cols(lane_base + c0 + q * 32, v[q]);
               tc_wait_ld();
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(t_empty(set));
             if (warp_live && r < a.rows) {
-              const int lim = min(first_pos + r % W, a.n - 1);    // last visible key of this row
-              float mx = -INFINITY;
+              if (tail) {
+                const int lim = min(first_pos + r % W, a.n - 1);  // last visible key of this row
 #pragma unroll
-              for (int q = 0; q < 4; ++q)
+                for (int q = 0; q < CW / 32; ++q)
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                  if (tail && key0 + q * 32 + e > lim) v[q][e] = -INFINITY;
-                  mx = fmaxf(mx, v[q][e]);
+                  for (int e = 0; e < 32; ++e)
+                    if (key0 + c0 + q * 32 + e > lim) v[q][e] = -INFINITY;
+              }
+              float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
+#pragma unroll
+              for (int q = 0; q < CW / 32; ++q)
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                  x0 = fmaxf(x0, v[q][e]);
+                  x1 = fmaxf(x1, v[q][e + 1]);
+                  x2 = fmaxf(x2, v[q][e + 2]);
+                  x3 = fmaxf(x3, v[q][e + 3]);
                 }
+              const float mx = fmaxf(fmaxf(x0, x1), fmaxf(x2, x3));
               float m_old = -INFINITY, l_old = 0.f;
 #pragma unroll
               for (int rb = 0; rb < kMaxRowBlocks; ++rb)
@@ -318,12 +339,14 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 const float mc = m_new * a.c;
                 float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                  s0 += ex2_approx(fmaf(v[0][e], a.c, -mc));
-                  s1 += ex2_approx(fmaf(v[1][e], a.c, -mc));
-                  s2 += ex2_approx(fmaf(v[2][e], a.c, -mc));
-                  s3 += ex2_approx(fmaf(v[3][e], a.c, -mc));
-                }
+                for (int q = 0; q < CW / 32; ++q)
+#pragma unroll
+                  for (int e = 0; e < 32; e += 4) {
+                    s0 += ex2_approx(fmaf(v[q][e], a.c, -mc));
+                    s1 += ex2_approx(fmaf(v[q][e + 1], a.c, -mc));
+                    s2 += ex2_approx(fmaf(v[q][e + 2], a.c, -mc));
+                    s3 += ex2_approx(fmaf(v[q][e + 3], a.c, -mc));
+                  }
                 l_old = l_old * ex2_approx((m_old - m_new) * a.c) + ((s0 + s1) + (s2 + s3));
                 m_old = m_new;
               }
@@ -335,26 +358,48 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             const int i = key0 + quad * 32 + lane;               // this thread's key
             const int h0 = sub * a.heads_per_group;
             const int nh = min(a.heads_per_group, a.G - h0);
-            for (int hq = 0; hq < nh; ++hq) {
+            const int hph = (a.heads_per_group + kHalves - 1) / kHalves;   // heads per column half
+            const int hq0 = half * hph, hq1 = min(nh, hq0 + hph);
+            if (hq0 >= hq1) {
+              tc_fence_before();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(t_empty(set));
+            }
+            for (int hq = hq0; hq < hq1; ++hq) {
               float v[W / 16][16];
 #pragma unroll
               for (int q = 0; q < W / 16; ++q) tmem_ld_16cols(lane_base + hq * W + q * 16, v[q]);
               tc_wait_ld();
-              if (hq == nh - 1) {
+              if (hq == hq1 - 1) {
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(t_empty(set));
               }
-              const float2* sr = st + (h0 + hq) * W;
-              float acc = 0.f;
+              // bias_j = -max_j * log2e + log2(1 / (w * sum_j)): one fma and one exp per weight
+              const float4* sr = reinterpret_cast<const float4*>(st + (h0 + hq) * W);
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+              if (!tail) {
 #pragma unroll
-              for (int j = 0; j < W; ++j) {
-                const float2 c2 = sr[j];
-                float p = ex2_approx(fmaf(v[j / 16][j % 16], a.c, c2.x)) * c2.y;
-                if (tail && i > first_pos + j) p = 0.f;
-                acc += p;
+                for (int j = 0; j < W; j += 4) {
+                  const float4 bz = sr[j / 4];
+                  a0 += ex2_approx(fmaf(v[j / 16][j % 16], a.c, bz.x));
+                  a1 += ex2_approx(fmaf(v[(j + 1) / 16][(j + 1) % 16], a.c, bz.y));
+                  a2 += ex2_approx(fmaf(v[(j + 2) / 16][(j + 2) % 16], a.c, bz.z));
+                  a3 += ex2_approx(fmaf(v[(j + 3) / 16][(j + 3) % 16], a.c, bz.w));
+                }
+              } else {
+                const int jmin = i - first_pos;                   // rows j < jmin do not see key i
+#pragma unroll
+                for (int j = 0; j < W; j += 4) {
+                  const float4 bz = sr[j / 4];
+                  a0 += j >= jmin ? ex2_approx(fmaf(v[j / 16][j % 16], a.c, bz.x)) : 0.f;
+                  a1 += j + 1 >= jmin ? ex2_approx(fmaf(v[(j + 1) / 16][(j + 1) % 16], a.c, bz.y)) : 0.f;
+                  a2 += j + 2 >= jmin ? ex2_approx(fmaf(v[(j + 2) / 16][(j + 2) % 16], a.c, bz.z)) : 0.f;
+                  a3 += j + 3 >= jmin ? ex2_approx(fmaf(v[(j + 3) / 16][(j + 3) % 16], a.c, bz.w)) : 0.f;
+                }
               }
-              if (i < a.n) a.abar[((long long)w.b * a.Hq + (long long)w.g * a.G + h0 + hq) * a.n + i] = acc;
+              if (i < a.n)
+                a.abar[((long long)w.b * a.Hq + (long long)w.g * a.G + h0 + hq) * a.n + i] = (a0 + a1) + (a2 + a3);
             }
           }
         }
@@ -369,7 +414,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
           const int r = rb * 128 + quad * 32 + lane;
           if (rb < a.row_blocks && r < a.rows) {
             const long long rowg = ((long long)w.b * a.Hq + (long long)w.g * a.G + r / W) * W + r % W;
-            const long long o = rowg * a.part_stride + w.chunk * 2 + set;
+            const long long o = rowg * a.part_stride + (w.chunk * 2 + set) * kHalves + half;
             a.part_m[o] = rm[rb] * a.scale;
             a.part_l[o] = rl[rb];
           }
@@ -440,11 +485,11 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
   const long long groups = (long long)d.nb * d.Hkv;
   long long want_items = 4LL * sm_count;
   int tpi = (int)((groups * a.ntiles + want_items - 1) / want_items);
-  if (tpi < 4) tpi = 4;
+  if (tpi < 4 * kHalves) tpi = 4 * kHalves;
   if (tpi > 64) tpi = 64;
   a.tiles_per_item = tpi;
   a.chunks_per_bg = (a.ntiles + tpi - 1) / tpi;
-  a.part_stride = 2 * a.chunks_per_bg;
+  a.part_stride = 2 * kHalves * a.chunks_per_bg;
   if (a.part_stride > (d.n + kAttnChunk - 1) / kAttnChunk + 2) return cudaErrorNotSupported;  // workspace layout
   a.nitems = groups * a.chunks_per_bg;
   a.scale = d.scale;
