@@ -137,6 +137,43 @@ def projection_norm(V, WO, *, rows=None, chunk=2048, norm="l1"):
     return nu
 
 
+def group_summed_projection(WO, G, storage="f32"):
+    """W_tilde [Hkv, dh, dm]: the output-projection slices of a KV group added up (float32, heads in increasing
+    order) and rounded once to the storage type.  Variant of step 2 for grouped-query attention: the heads of a
+    group share K and V, so their outputs add in o = sum_h A_h V_g W^O_h (Eq. 2 applied per head); projecting a
+    value row through the summed slice costs one contraction per KV head instead of one per query head.  The paper
+    does not spell this variant out; its memory figure for the projected values (one n x d matrix per KV head)
+    is consistent with it.  Returned widened to float32."""
+    WO = np.asarray(WO, dtype=F32)
+    Hq = WO.shape[0]
+    Hkv = Hq // G
+    out = np.empty((Hkv,) + WO.shape[1:], dtype=F32)
+    for g in range(Hkv):
+        acc = WO[g * G].copy()
+        for h in range(g * G + 1, (g + 1) * G):
+            acc = (acc + WO[h]).astype(F32)
+        out[g] = acc
+    if storage == "bf16":
+        import torch
+        out = torch.from_numpy(out).to(torch.bfloat16).to(torch.float32).numpy()
+    elif storage != "f32":
+        raise ValueError(storage)
+    return out
+
+
+def projection_norm_group_sum(V, WO, G, storage="f32", **kw):
+    """nu [Hkv, n]: L1 norm of each value row projected through its group's summed W^O slice."""
+    return projection_norm(V, group_summed_projection(WO, G, storage), **kw)
+
+
+def group_scores_group_sum(P, nu_g, G, eps=1e-4):
+    """a as in group_scores; c_g = (a_g + eps) * nu_g with nu_g [Hkv, n] (float32, separately rounded + and *)."""
+    a, _ = group_scores(P, np.ones_like(np.asarray(P, dtype=F32)), G, eps)
+    nu_g = np.asarray(nu_g).astype(F32)
+    c = ((a + F32(eps)).astype(F32) * nu_g).astype(F32)
+    return a, c
+
+
 # ----------------------------------------------------------------------------
 # Step 3: scores per KV head and budgets
 # (Algorithm 1: "A_cal = (A + eps) * row norms", "b' = b x alpha; b'' = b - b'";
@@ -220,13 +257,14 @@ def two_stage_select(a_g, c_g, b, alpha):
     return np.sort(S1), np.sort(S2)
 
 
-def select(P, nu, *, G, budget_mode, budget, alpha=0.5, eps=1e-4, budgets_in=None):
+def select(P, nu, *, G, budget_mode, budget, alpha=0.5, eps=1e-4, budgets_in=None, group_sum=False):
     """Steps 3+4 for one layer.
 
     Returns dict(idx [Btot] int32 packed by head, ascending inside a head;
     offsets [Hkv+1] int32; stage [Btot] uint8 (1 or 2); a, c float32; budgets).
+    group_sum: nu is [Hkv, n] from projection_norm_group_sum.
     """
-    a, c = group_scores(P, nu, G, eps)
+    a, c = group_scores_group_sum(P, nu, G, eps) if group_sum else group_scores(P, nu, G, eps)
     Hkv, n = a.shape
     if budget_mode == "given":
         budgets = np.asarray(budgets_in, dtype=np.int64)
@@ -261,12 +299,12 @@ def compact(K_store, V_store, idx, offsets):
 
 
 def compress_layer(Qw, K, V, WO, *, kp, budget_mode, budget, alpha=0.5, eps=1e-4, scale=None,
-                   K_store=None, V_store=None):
+                   K_store=None, V_store=None, group_sum=False, storage="f32"):
     """The whole path for one layer, step by step."""
     G = Qw.shape[0] // K.shape[0]
     P = pooled_window_attention(Qw, K, kp, scale)
-    nu = projection_norm(V, WO)
-    out = select(P, nu, G=G, budget_mode=budget_mode, budget=budget, alpha=alpha, eps=eps)
+    nu = projection_norm_group_sum(V, WO, G, storage) if group_sum else projection_norm(V, WO)
+    out = select(P, nu, G=G, budget_mode=budget_mode, budget=budget, alpha=alpha, eps=eps, group_sum=group_sum)
     Ko, Vo = compact(K if K_store is None else K_store, V if V_store is None else V_store,
                      out["idx"], out["offsets"])
     out.update(P=P, nu=nu, K_hat=Ko, V_hat=Vo)

@@ -173,6 +173,59 @@ def test_projection_norm_l2_variant():
     np.testing.assert_allclose(nu[0], ref, rtol=1e-12)
 
 
+def test_group_sum_projection_special_cases():
+    r = RNG(80)
+    Hkv, G, n, dh, dm = 2, 3, 6, 4, 5
+    V = r.standard_normal((Hkv, n, dh))
+    WO = r.standard_normal((Hkv * G, dh, dm)).astype(np.float32)
+    # a group of one head is the per-head norm
+    np.testing.assert_allclose(oc.projection_norm_group_sum(V, WO[:2], 1), oc.projection_norm(V, WO[:2]), rtol=1e-12)
+    # only one head of each group non-zero: that head's norm
+    W1 = np.zeros_like(WO)
+    W1[1], W1[5] = WO[1], WO[5]
+    nu = oc.projection_norm_group_sum(V, W1, G)
+    np.testing.assert_allclose(nu, oc.projection_norm(V, W1)[[1, 5]], rtol=1e-12)
+    # opposite slices cancel before the norm is taken (a sum of per-head norms would not)
+    W2 = np.zeros_like(WO)
+    W2[0], W2[1] = WO[0], -WO[0]
+    assert np.all(oc.projection_norm_group_sum(V, W2, G)[0] == 0)
+    # scaled identities: nu = |sum of scales| * ||v||_1
+    W3 = np.zeros((G, dh, dm), np.float32)
+    for h, sc in enumerate((0.5, -2.0, 4.0)):
+        W3[h, np.arange(dh), np.arange(dh)] = sc
+    np.testing.assert_allclose(oc.projection_norm_group_sum(V[:1], W3, G)[0], 2.5 * np.abs(V[0]).sum(axis=1), rtol=1e-12)
+    # triple loop
+    nu = oc.projection_norm_group_sum(V, WO, G)
+    for g in range(Hkv):
+        for i in range(n):
+            tot = 0.0
+            for c in range(dm):
+                tot += abs(sum(V[g, i, t] * sum(float(WO[g * G + q, t, c]) for q in range(G)) for t in range(dh)))
+            assert abs(nu[g, i] - tot) < 1e-5 * tot          # float32 sums of the slices
+
+
+def test_group_sum_projection_rounds_once_to_bf16():
+    import torch
+    r = RNG(81)
+    WO = torch.from_numpy(r.standard_normal((4, 3, 8)).astype(np.float32)).to(torch.bfloat16).to(torch.float32).numpy()
+    Wt = oc.group_summed_projection(WO, 4, "bf16")
+    exact = WO.astype(np.float64).sum(axis=0)
+    assert np.all(np.abs(Wt[0] - exact) <= 2.0 ** -8 * np.abs(exact) + 1e-30)                  # one bf16 rounding
+    assert np.array_equal(Wt, torch.from_numpy(Wt).to(torch.bfloat16).to(torch.float32).numpy())  # representable
+
+
+def test_group_sum_scores():
+    r = RNG(82)
+    P = r.random((6, 20)).astype(np.float32)
+    nu = (r.random((2, 20)) * 9).astype(np.float32)
+    a, c = oc.group_scores_group_sum(P, nu, 3, 1e-4)
+    a_ref, _ = oc.group_scores(P, np.ones_like(P), 3)
+    np.testing.assert_array_equal(a, a_ref)
+    np.testing.assert_allclose(c, (P.reshape(2, 3, -1).mean(axis=1) + 1e-4) * nu, rtol=1e-6)
+    out = oc.select(P, nu, G=3, budget_mode="uniform", budget=5, group_sum=True)
+    assert out["idx"].size == 10
+
+
 # ----------------------------------------------------------------------------- step 3
 def test_group_scores_special_cases():
     r = RNG(9)
