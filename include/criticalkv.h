@@ -66,7 +66,13 @@ typedef enum { CKV_NORM_L1 = 0 } criticalkv_norm;
 
 enum {
   CKV_FLAG_WO_SHARED = 1u << 0,   /* WO has no nb dimension (one projection for the whole call)             */
-  CKV_FLAG_FORCE_SIMT = 1u << 1   /* bf16 only: use the CUDA-core kernels instead of the tensor-core ones   */
+  CKV_FLAG_FORCE_SIMT = 1u << 1,  /* bf16 only: use the CUDA-core kernels instead of the tensor-core ones   */
+  CKV_FLAG_WO_GROUP_SUM = 1u << 2 /* grouped-query shortcut of step 2: the W^O slices of a KV group are added
+                                     (float32, heads ascending, rounded once to the storage type) and each value
+                                     row is projected once per KV head.  vnorm then is [nb, Hkv, n] and
+                                     c_g = (a_g + eps) * vnorm_g in criticalkv_select.  Hq/Hkv times fewer flops;
+                                     not the per-head norm of Algorithm 1 but the norm of the group's summed
+                                     projection (the heads of a group share V, so their outputs add in Eq. 2).  */
 };
 
 /* Problem descriptor (plain data, copied by every call). */

@@ -18,7 +18,7 @@ CKV_OK, CKV_EINVAL, CKV_ENOTSUP, CKV_EALIGN, CKV_EWORKSPACE, CKV_ECUDA, CKV_ETIM
 CKV_F32, CKV_BF16 = 0, 1
 CKV_BUDGET_UNIFORM, CKV_BUDGET_FLAT_ADAPTIVE, CKV_BUDGET_GIVEN = 0, 1, 2
 CKV_NORM_L1 = 0
-CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT = 1, 2
+CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM = 1, 2, 4
 CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",

@@ -53,7 +53,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (!(d->eps >= 0.f) || !isfinite(d->eps)) return CKV_EINVAL;
   if (d->norm != CKV_NORM_L1) return CKV_ENOTSUP;
   if (d->reserved != 0) return CKV_EINVAL;
-  if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT)) return CKV_EINVAL;
+  if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM)) return CKV_EINVAL;
   if (d->budget < 0) return CKV_EINVAL;
   if ((long long)d->n * d->Hkv > 0x7fffffffLL) return CKV_ENOTSUP;
   o->nb = d->nb; o->Hq = d->Hq; o->Hkv = d->Hkv; o->G = d->Hq / d->Hkv;
@@ -76,6 +76,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   }
   if (o->btot > 0x7fffffffLL) return CKV_ENOTSUP;
   o->wo_shared = (d->flags & CKV_FLAG_WO_SHARED) ? 1 : 0;
+  o->group_sum = (d->flags & CKV_FLAG_WO_GROUP_SUM) ? 1 : 0;
   const long long dq[3] = {(long long)d->Hq * d->w * d->dh, (long long)d->w * d->dh, d->dh};
   const long long dk[3] = {(long long)d->Hkv * d->n * d->dh, (long long)d->n * d->dh, d->dh};
   const int vec = d->dtype == CKV_F32 ? 4 : 8;  // elements per 16 bytes
@@ -91,7 +92,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
 }
 
 struct ScoreLayout {
-  size_t part_m, part_l, rowstat, abar, total;
+  size_t part_m, part_l, rowstat, abar, wsum, total;
 };
 ScoreLayout score_layout(const Dims& d) {
   ScoreLayout L;
@@ -104,6 +105,9 @@ ScoreLayout score_layout(const Dims& d) {
   L.part_l = off; off = align_up(off + rows * nchunks * sizeof(float), 256);
   L.rowstat = off; off = align_up(off + rows * 2 * sizeof(float), 256);
   L.abar = off; off = align_up(off + (size_t)d.nb * d.Hq * d.n * sizeof(float), 256);
+  L.wsum = off;
+  if (d.group_sum)
+    off = align_up(off + (size_t)(d.wo_shared ? 1 : d.nb) * d.Hkv * d.dh * d.dm * (d.dtype == CKV_F32 ? 4 : 2), 256);
   L.total = off;
   return L;
 }
@@ -203,7 +207,7 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
   cudaStream_t st = (cudaStream_t)stream;
   char* base = (char*)ws;
   ckv::ScoreWorkspace sw{(float*)(base + L.part_m), (float*)(base + L.part_l), (float*)(base + L.rowstat),
-                         (float*)(base + L.abar)};
+                         (float*)(base + L.abar), (void*)(base + L.wsum)};
   int launches = 0, path = 0;
   cudaError_t e = cudaSuccess;
   if (attn) {
@@ -221,6 +225,13 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
       e = ckv::launch_window_attn_simt(dd, Qw, K, attn, sw, st, &launches);
       path |= 4;
     }
+  }
+  if (e == cudaSuccess && vnorm && dd.group_sum) {
+    // one projection per KV head through the group's summed W^O slice: same kernels, seen as Hkv heads of group size 1
+    e = ckv::launch_wo_group_sum(dd, WO, sw.wsum, st, &launches);
+    WO = sw.wsum;
+    dd.Hq = dd.Hkv;
+    dd.G = 1;
   }
   if (e == cudaSuccess && vnorm) {
     bool done = false;

@@ -16,6 +16,7 @@ struct Dims {
   long long budget;   // as in criticalkv_desc
   long long btot;     // capacity of idx per nb slice
   int wo_shared;
+  int group_sum;      // CKV_FLAG_WO_GROUP_SUM
   long long qs[3], ks[3], vs[3];  // element strides: nb, head, row
 };
 
@@ -27,6 +28,7 @@ struct ScoreWorkspace {   // carved out of the caller's workspace by the API lay
   float* part_l;    // [nb*Hq*w, nchunks]   partial row sums of exp
   float* rowstat;   // [nb*Hq*w, 2]         final (max, 1/(w*sum))
   float* abar;      // [nb*Hq, n]           window-mean attention before pooling
+  void* wsum;       // [nbw, Hkv, dh, dm]   group-summed W^O (CKV_FLAG_WO_GROUP_SUM only)
 };
 
 struct SelectWorkspace {
@@ -54,6 +56,8 @@ cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, floa
                               int* status_word, cudaStream_t st, int* launches);
 cudaError_t launch_bounded_wait_selftest(int* status_word, unsigned long long limit_ns, int* observed,
                                          cudaStream_t st);
+// W_tilde[bw, g] = round(sum_h WO[bw, g*G + h]) for the group-summed projection variant.
+cudaError_t launch_wo_group_sum(const Dims& d, const void* WO, void* wsum, cudaStream_t st, int* launches);
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word);

@@ -24,21 +24,31 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 __global__ void group_reduce_kernel(const float* __restrict__ attn, const float* __restrict__ vnorm,
                                     float* __restrict__ a, float* __restrict__ c, int Hq, int Hkv, int G, int n,
-                                    float eps) {
+                                    float eps, int group_sum) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int g = blockIdx.y, b = blockIdx.z;
   const long long h0 = (long long)b * Hq + (long long)g * G;
-  float p = attn[h0 * n + i];
-  float sa = p;
-  float sc = __fmul_rn(__fadd_rn(p, eps), vnorm[h0 * n + i]);
-  for (int q = 1; q < G; ++q) {
-    p = attn[(h0 + q) * n + i];
-    sa = __fadd_rn(sa, p);
-    sc = __fadd_rn(sc, __fmul_rn(__fadd_rn(p, eps), vnorm[(h0 + q) * n + i]));
-  }
   const float Gf = (float)G;
-  float av = __fdiv_rn(sa, Gf), cv = __fdiv_rn(sc, Gf);
+  float av, cv;
+  if (group_sum) {
+    // vnorm is per KV head: c = (a + eps) * nu_g
+    float sa = attn[h0 * n + i];
+    for (int q = 1; q < G; ++q) sa = __fadd_rn(sa, attn[(h0 + q) * n + i]);
+    av = __fdiv_rn(sa, Gf);
+    cv = __fmul_rn(__fadd_rn(av, eps), vnorm[((long long)b * Hkv + g) * n + i]);
+  } else {
+    float p = attn[h0 * n + i];
+    float sa = p;
+    float sc = __fmul_rn(__fadd_rn(p, eps), vnorm[h0 * n + i]);
+    for (int q = 1; q < G; ++q) {
+      p = attn[(h0 + q) * n + i];
+      sa = __fadd_rn(sa, p);
+      sc = __fadd_rn(sc, __fmul_rn(__fadd_rn(p, eps), vnorm[(h0 + q) * n + i]));
+    }
+    av = __fdiv_rn(sa, Gf);
+    cv = __fdiv_rn(sc, Gf);
+  }
   if (av == 0.f) av = 0.f;  // -0 and +0 must order alike
   if (cv == 0.f) cv = 0.f;
   const long long o = ((long long)b * Hkv + g) * n + i;
@@ -273,7 +283,7 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word) {
   dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
-  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, ws.a, ws.c, d.Hq, d.Hkv, d.G, d.n, d.eps);
+  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, ws.a, ws.c, d.Hq, d.Hkv, d.G, d.n, d.eps, d.group_sum);
   *launches += 1;
   const int32_t* budgets = nullptr;
   if (d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {

@@ -84,6 +84,19 @@ __global__ void __launch_bounds__(kThreads) vnorm_simt_kernel(VnormArgs a) {
   }
 }
 
+// out[bw, g, :] = round_to_T(W[bw, g*G] + W[bw, g*G+1] + ...) in float32, heads in increasing order.
+template <typename T>
+__global__ void wo_group_sum_kernel(const T* __restrict__ W, T* __restrict__ out, int G, long long per_head,
+                                    long long total) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // element of out
+  if (e >= total) return;
+  const long long grp = e / per_head, r = e % per_head;
+  const T* src = W + grp * G * per_head + r;
+  float acc = ldf(src);
+  for (int q = 1; q < G; ++q) acc = __fadd_rn(acc, ldf(src + q * per_head));
+  out[e] = T(acc);
+}
+
 template <typename T, int DH>
 cudaError_t run(const Dims& d, const VnormArgs& a, cudaStream_t st, int* launches) {
   const size_t smem = (size_t)(DH * (BM + PAD) + DH * BN) * sizeof(float);
@@ -97,6 +110,19 @@ cudaError_t run(const Dims& d, const VnormArgs& a, cudaStream_t st, int* launche
 }
 
 }  // namespace
+
+cudaError_t launch_wo_group_sum(const Dims& d, const void* WO, void* wsum, cudaStream_t st, int* launches) {
+  const long long per_head = (long long)d.dh * d.dm;
+  const long long total = (long long)(d.wo_shared ? 1 : d.nb) * d.Hkv * per_head;
+  const unsigned blocks = (unsigned)((total + 255) / 256);
+  if (d.dtype == CKV_F32)
+    wo_group_sum_kernel<float><<<blocks, 256, 0, st>>>((const float*)WO, (float*)wsum, d.G, per_head, total);
+  else
+    wo_group_sum_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>((const __nv_bfloat16*)WO, (__nv_bfloat16*)wsum, d.G,
+                                                              per_head, total);
+  *launches += 1;
+  return cudaGetLastError();
+}
 
 cudaError_t launch_vnorm_simt(const Dims& d, const void* V, const void* WO, float* vnorm, cudaStream_t st,
                               int* launches) {

@@ -44,7 +44,8 @@ class CompressionSession:
         self.score_bytes, self.select_bytes = sb, tb
         self.ws = torch.empty(max(sb, tb, 256), dtype=torch.uint8, device=dev)
         self.attn = torch.empty((nb, Hq, n), dtype=torch.float32, device=dev)
-        self.vnorm = torch.empty((nb, Hq, n), dtype=torch.float32, device=dev)
+        self.vnorm = torch.empty((nb, Hkv if flags & B.CKV_FLAG_WO_GROUP_SUM else Hq, n), dtype=torch.float32,
+                                 device=dev)
         self.idx = torch.full((nb, max(self.btot, 1)), -1, dtype=torch.int32, device=dev)
         self.offsets = torch.zeros((nb, Hkv + 1), dtype=torch.int32, device=dev)
         self.stage = torch.zeros((nb, max(self.btot, 1)), dtype=torch.uint8, device=dev) if want_stage else None

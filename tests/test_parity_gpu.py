@@ -197,6 +197,26 @@ def test_host_staged_compress_equals_device_compress(mode, budget, shared):
         np.testing.assert_array_equal(to_host(Vo[b])[:tot], to_host(s.V_out[0])[:tot])
 
 
+@pytest.mark.parametrize("kw", [
+    dict(dtype="bf16", n=1300, w=32, kp=7, budget=180, dh=128, dm=512, Hq=8, Hkv=2),
+    dict(dtype="f32", n=500, w=16, kp=5, budget=70, dh=64, dm=192, Hq=6, Hkv=2),
+    dict(dtype="bf16", n=2100, w=32, kp=7, budget_mode="adaptive", budget=900, dh=128, dm=1024, Hq=16, Hkv=4),
+])
+def test_group_summed_projection_variant(kw):
+    # CKV_FLAG_WO_GROUP_SUM: one projection per KV head through the summed W^O slices of its group
+    from paper_2502_03805_b200 import binding as B
+    wl = small_workload(cfg_id=170, **kw)
+    Ls, outs, s = _run(wl, layers=(0, 1), flags=B.CKV_FLAG_WO_GROUP_SUM)
+    assert outs[0]["vnorm"].shape == (wl.Hkv, wl.n)
+    if wl.dtype == "bf16":
+        assert s.last_path == 3
+    for L, out in zip(Ls, outs):
+        pu.check_layer_against_oracle(L, wl, out, group_sum=True)
+    # and it is a different quantity from the per-head norm unless the group has one head
+    _, std, _ = _run(wl, layers=(0,))
+    assert not np.allclose(std[0]["vnorm"][:: wl.G], outs[0]["vnorm"], rtol=1e-2)
+
+
 def test_bounded_wait_times_out_and_reports_status():
     # a wait on a barrier nothing signals must end by itself, set CKV_ETIMEOUT, and leave the context usable
     import time
