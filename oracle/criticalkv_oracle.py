@@ -224,21 +224,38 @@ def stable_topk(x, k):
     return order[:k]
 
 
-def allocate_budgets(a, mode, budget):
+def allocate_budgets(a, mode, budget, floor=0.0):
     """Per-KV-head budgets b_g (Algorithm 2, budget allocation step).
 
     uniform : every head gets ``budget``.
     adaptive: the ``budget`` largest entries of the flattened [Hkv * n]
               attention scores are counted per head (ties: lower flattened
               index g * n + i first).
+    floor   : adaptive only.  Every head is first guaranteed
+              floor_b = floor(floor * budget / Hkv) entries (the safeguard of
+              adaptive allocation schemes), the remaining budget - Hkv * floor_b
+              entries are allocated by the flattened top-k, and b_g is capped at n.
     """
     Hkv, n = a.shape
     if mode == "uniform":
         return np.full(Hkv, int(budget), dtype=np.int64)
     if mode == "adaptive":
-        top = stable_topk(a.reshape(-1), int(budget))
-        return np.bincount(top // n, minlength=Hkv).astype(np.int64)
+        floor_b = int(math.floor(float(F32(floor)) * float(budget) / float(Hkv)))
+        floor_b = min(max(floor_b, 0), int(budget) // Hkv)
+        top = stable_topk(a.reshape(-1), int(budget) - Hkv * floor_b)
+        counts = np.bincount(top // n, minlength=Hkv).astype(np.int64)
+        return np.minimum(counts + floor_b, n)
     raise ValueError(mode)
+
+
+def protect_window(a, c, w):
+    """Variant: the last w entries (the observation window itself) are always kept.  Their scores are raised to the
+    largest float32 in both stages, so they fill stage 1 first (lowest index first) and count against the budget."""
+    a, c = a.copy(), c.copy()
+    big = np.finfo(F32).max
+    a[:, a.shape[1] - w:] = big
+    c[:, c.shape[1] - w:] = big
+    return a, c
 
 
 # ----------------------------------------------------------------------------
@@ -257,7 +274,8 @@ def two_stage_select(a_g, c_g, b, alpha):
     return np.sort(S1), np.sort(S2)
 
 
-def select(P, nu, *, G, budget_mode, budget, alpha=0.5, eps=1e-4, budgets_in=None, group_sum=False):
+def select(P, nu, *, G, budget_mode, budget, alpha=0.5, eps=1e-4, budgets_in=None, group_sum=False,
+           adaptive_floor=0.0, protect_w=0):
     """Steps 3+4 for one layer.
 
     Returns dict(idx [Btot] int32 packed by head, ascending inside a head;
@@ -265,11 +283,13 @@ def select(P, nu, *, G, budget_mode, budget, alpha=0.5, eps=1e-4, budgets_in=Non
     group_sum: nu is [Hkv, n] from projection_norm_group_sum.
     """
     a, c = group_scores_group_sum(P, nu, G, eps) if group_sum else group_scores(P, nu, G, eps)
+    if protect_w:
+        a, c = protect_window(a, c, protect_w)
     Hkv, n = a.shape
     if budget_mode == "given":
         budgets = np.asarray(budgets_in, dtype=np.int64)
     else:
-        budgets = allocate_budgets(a, budget_mode, budget)
+        budgets = allocate_budgets(a, budget_mode, budget, adaptive_floor)
     idx, stage, offsets = [], [], [0]
     for g in range(Hkv):
         S1, S2 = two_stage_select(a[g], c[g], int(budgets[g]), alpha)

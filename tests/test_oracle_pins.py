@@ -293,6 +293,40 @@ def test_adaptive_budgets():
     assert list(oc.allocate_budgets(a, "uniform", 9)) == [9] * Hkv
 
 
+def test_adaptive_floor():
+    r = RNG(83)
+    Hkv, n, B = 4, 50, 80
+    a = r.random((Hkv, n)).astype(np.float32)
+    a[0] *= 10                                            # head 0 would take almost everything
+    plain = oc.allocate_budgets(a, "adaptive", B)
+    assert plain.sum() == B and plain[0] >= 40 and plain[1:].min() < 15
+    half = oc.allocate_budgets(a, "adaptive", B, floor=0.5)
+    assert half.min() >= 10                               # floor(0.5 * 80 / 4) guaranteed per head
+    rest = oc.allocate_budgets(a, "adaptive", B - 4 * 10)
+    np.testing.assert_array_equal(half, np.minimum(rest + 10, n))
+    full = oc.allocate_budgets(a, "adaptive", B, floor=1.0)
+    assert list(full) == [20, 20, 20, 20]                 # floor 1 is the uniform split
+    np.testing.assert_array_equal(oc.allocate_budgets(a, "adaptive", B, floor=0.0), plain)
+
+
+def test_protect_window_keeps_the_last_w_entries():
+    r = RNG(84)
+    Hq, G, n, w = 4, 2, 40, 6
+    P = r.random((Hq, n))
+    P[:, n - w:] = 0.0                                    # the window would otherwise be dropped
+    nu = np.exp(r.standard_normal((Hq, n)))
+    for mode, budget in (("uniform", 10), ("adaptive", 24)):
+        out = oc.select(P, nu, G=G, budget_mode=mode, budget=budget, protect_w=w)
+        base = oc.select(P, nu, G=G, budget_mode=mode, budget=budget)
+        for g in range(2):
+            seg = out["idx"][out["offsets"][g]:out["offsets"][g + 1]]
+            assert set(range(n - w, n)) <= set(seg.tolist())
+            assert not set(range(n - w, n)) & set(base["idx"][base["offsets"][g]:base["offsets"][g + 1]].tolist())
+    # a budget smaller than the window keeps its first entries (lowest index first)
+    tiny = oc.select(P, nu, G=G, budget_mode="uniform", budget=4, protect_w=w)
+    assert tiny["idx"][:4].tolist() == [n - w, n - w + 1, n - w + 2, n - w + 3]
+
+
 # ----------------------------------------------------------------------------- step 4
 def _scores(seed, n=40, dup=False):
     r = RNG(seed)
