@@ -67,6 +67,9 @@ typedef enum { CKV_NORM_L1 = 0 } criticalkv_norm;
 enum {
   CKV_FLAG_WO_SHARED = 1u << 0,   /* WO has no nb dimension (one projection for the whole call)             */
   CKV_FLAG_FORCE_SIMT = 1u << 1,  /* bf16 only: use the CUDA-core kernels instead of the tensor-core ones   */
+  CKV_FLAG_PROTECT_WINDOW = 1u << 3, /* always keep the last w entries (the observation window): their scores are
+                                     raised to the largest float32 in both stages, so they fill stage 1 first and
+                                     count against the budget                                                   */
   CKV_FLAG_WO_GROUP_SUM = 1u << 2 /* grouped-query shortcut of step 2: the W^O slices of a KV group are added
                                      (float32, heads ascending, rounded once to the storage type) and each value
                                      row is projected once per KV head.  vnorm then is [nb, Hkv, n] and
@@ -98,6 +101,10 @@ typedef struct {
   int64_t q_stride[3];
   int64_t k_stride[3];
   int64_t v_stride[3];
+  float adaptive_floor;  /* FLAT_ADAPTIVE only, in [0,1]: every KV head is first guaranteed
+                            floor(adaptive_floor * budget / Hkv) entries, the rest of the budget goes to the
+                            flattened top-k, and a head's budget is capped at n.  0 in the paper's settings.   */
+  uint32_t reserved2;    /* must be 0                                                                   */
 } criticalkv_desc;
 
 /* Create / destroy a handle bound to CUDA device `device`.  create allocates one device status word. */

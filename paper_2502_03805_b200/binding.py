@@ -18,7 +18,7 @@ CKV_OK, CKV_EINVAL, CKV_ENOTSUP, CKV_EALIGN, CKV_EWORKSPACE, CKV_ECUDA, CKV_ETIM
 CKV_F32, CKV_BF16 = 0, 1
 CKV_BUDGET_UNIFORM, CKV_BUDGET_FLAT_ADAPTIVE, CKV_BUDGET_GIVEN = 0, 1, 2
 CKV_NORM_L1 = 0
-CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM = 1, 2, 4
+CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM, CKV_FLAG_PROTECT_WINDOW = 1, 2, 4, 8
 CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",
@@ -34,7 +34,8 @@ class criticalkv_desc(C.Structure):
                 ("scale", C.c_float), ("alpha", C.c_float), ("eps", C.c_float),
                 ("budget_mode", C.c_int32), ("norm", C.c_int32), ("budget", C.c_int64),
                 ("flags", C.c_uint32), ("reserved", C.c_uint32),
-                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3), ("v_stride", C.c_int64 * 3)]
+                ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3), ("v_stride", C.c_int64 * 3),
+                ("adaptive_floor", C.c_float), ("reserved2", C.c_uint32)]
 
 
 class CriticalKVError(RuntimeError):
@@ -109,7 +110,8 @@ def status_string(status: int) -> str:
 
 
 def make_desc(*, nb, Hq, Hkv, dh, dm, n, w, pool_k, dtype, budget_mode, budget, alpha=0.5, eps=1e-4, scale=0.0,
-              flags=0, norm=CKV_NORM_L1, q_stride=(0, 0, 0), k_stride=(0, 0, 0), v_stride=(0, 0, 0)):
+              flags=0, norm=CKV_NORM_L1, q_stride=(0, 0, 0), k_stride=(0, 0, 0), v_stride=(0, 0, 0),
+              adaptive_floor=0.0):
     d = criticalkv_desc()
     d.nb, d.Hq, d.Hkv, d.dh, d.dm, d.n, d.w, d.pool_k = nb, Hq, Hkv, dh, dm, n, w, pool_k
     d.dtype = {"f32": CKV_F32, "bf16": CKV_BF16}.get(dtype, dtype)
@@ -120,6 +122,7 @@ def make_desc(*, nb, Hq, Hkv, dh, dm, n, w, pool_k, dtype, budget_mode, budget, 
     d.q_stride[:] = q_stride
     d.k_stride[:] = k_stride
     d.v_stride[:] = v_stride
+    d.adaptive_floor, d.reserved2 = adaptive_floor, 0
     return d
 
 

@@ -52,8 +52,10 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (!(d->alpha >= 0.f && d->alpha <= 1.f)) return CKV_EINVAL;
   if (!(d->eps >= 0.f) || !isfinite(d->eps)) return CKV_EINVAL;
   if (d->norm != CKV_NORM_L1) return CKV_ENOTSUP;
-  if (d->reserved != 0) return CKV_EINVAL;
-  if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM)) return CKV_EINVAL;
+  if (d->reserved != 0 || d->reserved2 != 0) return CKV_EINVAL;
+  if (!(d->adaptive_floor >= 0.f && d->adaptive_floor <= 1.f)) return CKV_EINVAL;
+  if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM |
+                             CKV_FLAG_PROTECT_WINDOW)) return CKV_EINVAL;
   if (d->budget < 0) return CKV_EINVAL;
   if ((long long)d->n * d->Hkv > 0x7fffffffLL) return CKV_ENOTSUP;
   o->nb = d->nb; o->Hq = d->Hq; o->Hkv = d->Hkv; o->G = d->Hq / d->Hkv;
@@ -77,6 +79,13 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (o->btot > 0x7fffffffLL) return CKV_ENOTSUP;
   o->wo_shared = (d->flags & CKV_FLAG_WO_SHARED) ? 1 : 0;
   o->group_sum = (d->flags & CKV_FLAG_WO_GROUP_SUM) ? 1 : 0;
+  o->protect_window = (d->flags & CKV_FLAG_PROTECT_WINDOW) ? 1 : 0;
+  o->floor_b = 0;
+  if (d->budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
+    long long fb = (long long)floor((double)d->adaptive_floor * (double)d->budget / (double)d->Hkv);
+    const long long cap = d->budget / d->Hkv;
+    o->floor_b = fb < 0 ? 0 : (fb > cap ? cap : fb);
+  }
   const long long dq[3] = {(long long)d->Hq * d->w * d->dh, (long long)d->w * d->dh, d->dh};
   const long long dk[3] = {(long long)d->Hkv * d->n * d->dh, (long long)d->n * d->dh, d->dh};
   const int vec = d->dtype == CKV_F32 ? 4 : 8;  // elements per 16 bytes

@@ -17,6 +17,8 @@ struct Dims {
   long long btot;     // capacity of idx per nb slice
   int wo_shared;
   int group_sum;      // CKV_FLAG_WO_GROUP_SUM
+  int protect_window; // CKV_FLAG_PROTECT_WINDOW
+  long long floor_b;  // guaranteed entries per KV head (adaptive budgets)
   long long qs[3], ks[3], vs[3];  // element strides: nb, head, row
 };
 

@@ -24,7 +24,7 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 __global__ void group_reduce_kernel(const float* __restrict__ attn, const float* __restrict__ vnorm,
                                     float* __restrict__ a, float* __restrict__ c, int Hq, int Hkv, int G, int n,
-                                    float eps, int group_sum) {
+                                    float eps, int group_sum, int protect_from) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int g = blockIdx.y, b = blockIdx.z;
@@ -49,6 +49,7 @@ __global__ void group_reduce_kernel(const float* __restrict__ attn, const float*
     av = __fdiv_rn(sa, Gf);
     cv = __fdiv_rn(sc, Gf);
   }
+  if (i >= protect_from) av = cv = 3.402823466e+38f;  // protected observation window: largest float32
   if (av == 0.f) av = 0.f;  // -0 and +0 must order alike
   if (cv == 0.f) cv = 0.f;
   const long long o = ((long long)b * Hkv + g) * n + i;
@@ -238,14 +239,14 @@ __global__ void __launch_bounds__(kSelThreads) two_stage_kernel(TwoStageArgs p) 
 // Flattened top-B_total over a[nb, Hkv*n]: budgets[g] = #{i : key > T} + the first ties in (g, i) order.
 __global__ void __launch_bounds__(kSelThreads) adaptive_budget_kernel(const float* __restrict__ a,
                                                                       int32_t* __restrict__ budgets, int Hkv, int n,
-                                                                      long long btotal) {
+                                                                      long long btotal, int floor_b) {
   __shared__ SelectShared sh;
   __shared__ uint32_t cnt_gt[64], cnt_eq[64];
   const int b = blockIdx.x;
   const float* ab = a + (long long)b * Hkv * n;
   int32_t* out = budgets + (long long)b * Hkv;
-  if (btotal <= 0) {
-    if (threadIdx.x < Hkv) out[threadIdx.x] = 0;
+  if (btotal <= 0) {  // nothing left for the flattened top-k: every head gets its guaranteed share
+    if (threadIdx.x < Hkv) out[threadIdx.x] = min(floor_b, n);
     return;
   }
   uint32_t T, r;
@@ -271,7 +272,7 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_kernel(const floa
     uint32_t rem = r;
     for (int g = 0; g < Hkv; ++g) {
       const uint32_t take = min(cnt_eq[g], rem);
-      out[g] = (int32_t)(cnt_gt[g] + take);
+      out[g] = (int32_t)min((long long)cnt_gt[g] + take + floor_b, (long long)n);
       rem -= take;
     }
   }
@@ -283,11 +284,13 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word) {
   dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
-  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, ws.a, ws.c, d.Hq, d.Hkv, d.G, d.n, d.eps, d.group_sum);
+  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, ws.a, ws.c, d.Hq, d.Hkv, d.G, d.n, d.eps, d.group_sum,
+                                             d.protect_window ? d.n - d.w : d.n);
   *launches += 1;
   const int32_t* budgets = nullptr;
   if (d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
-    adaptive_budget_kernel<<<d.nb, kSelThreads, 0, st>>>(ws.a, ws.budgets, d.Hkv, d.n, d.budget);
+    adaptive_budget_kernel<<<d.nb, kSelThreads, 0, st>>>(ws.a, ws.budgets, d.Hkv, d.n, d.budget - d.Hkv * d.floor_b,
+                                                         (int)d.floor_b);
     *launches += 1;
     budgets = ws.budgets;
   } else if (d.budget_mode == CKV_BUDGET_GIVEN) {

@@ -217,6 +217,30 @@ def test_group_summed_projection_variant(kw):
     assert not np.allclose(std[0]["vnorm"][:: wl.G], outs[0]["vnorm"], rtol=1e-2)
 
 
+@pytest.mark.parametrize("floor", [0.0, 0.3, 1.0])
+@pytest.mark.parametrize("protect", [False, True])
+def test_adaptive_floor_and_protected_window_are_bit_exact_on_identical_scores(floor, protect):
+    from paper_2502_03805_b200 import binding as B, session_for
+    r = np.random.default_rng(9)
+    Hq, Hkv, n, w, budget = 8, 4, 900, 8, 700
+    P = r.random((Hq, n)).astype(np.float32) ** 6
+    P[:4] *= 20                                               # two heads would take nearly everything
+    P[:, n - w:] *= 1e-3
+    nu = np.exp(r.standard_normal((Hq, n))).astype(np.float32)
+    wl = small_workload(cfg_id=142, Hq=Hq, Hkv=Hkv, n=n, w=w, budget_mode="adaptive", budget=budget)
+    ref = oc.select(P, nu, G=2, budget_mode="adaptive", budget=budget, adaptive_floor=floor,
+                    protect_w=w if protect else 0)
+    s = session_for(wl, nb=1, adaptive_floor=floor, flags=B.CKV_FLAG_PROTECT_WINDOW if protect else 0)
+    s.select(torch.from_numpy(P)[None].cuda(), torch.from_numpy(nu)[None].cuda())
+    torch.cuda.synchronize()
+    off = s.offsets[0].cpu().numpy()
+    np.testing.assert_array_equal(off, ref["offsets"])
+    np.testing.assert_array_equal(s.idx[0].cpu().numpy()[: off[-1]], ref["idx"])
+    np.testing.assert_array_equal(s.stage[0].cpu().numpy()[: off[-1]], ref["stage"])
+    if floor == 1.0:
+        assert list(np.diff(off)) == [budget // Hkv] * Hkv
+
+
 def test_bounded_wait_times_out_and_reports_status():
     # a wait on a barrier nothing signals must end by itself, set CKV_ETIMEOUT, and leave the context usable
     import time
