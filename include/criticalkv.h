@@ -164,6 +164,15 @@ CKV_API int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc*
 CKV_API int criticalkv_compact(criticalkv_handle h, const criticalkv_desc* d, const void* K, const void* V,
                                const int32_t* idx, const int32_t* offsets, void* K_out, void* V_out, void* stream);
 
+/*
+ * Companion of criticalkv_compact for chunked prefill (the paper's long-context deployment: the cache is compressed
+ * after every prefill chunk and later chunks see [retained entries ; new chunk]).  pos_in[nb,Hkv,n] int32 holds the
+ * original token position of every cached entry; pos_out[nb, r] = pos_in[nb, g, idx[nb, r]] keeps them attached to
+ * the retained rows.
+ */
+CKV_API int criticalkv_gather_positions(criticalkv_handle h, const criticalkv_desc* d, const int32_t* pos_in,
+                                        const int32_t* idx, const int32_t* offsets, int32_t* pos_out, void* stream);
+
 /* The three calls above back to back on one stream.  ws must hold max(score_bytes, select_bytes). */
 CKV_API int criticalkv_compress(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K,
                                 const void* V, const void* WO, const int32_t* budgets_in, float* attn, float* vnorm,

@@ -331,6 +331,39 @@ def compress_layer(Qw, K, V, WO, *, kp, budget_mode, budget, alpha=0.5, eps=1e-4
     return out
 
 
+def chunked_compress(chunks, WO, *, kp, w, budgets, alpha=0.5, eps=1e-4, scale=None):
+    """Chunked prefill with eviction between chunks (the paper's long-context deployment, appendix on chunked
+    prefill): for every chunk the cache is [retained entries ; the chunk's K, V], the observation window is the last
+    w queries of the chunk, and the cache is compressed to ``budgets[c]`` entries per KV head (uniform budgets, so
+    every head keeps the same number).  Later chunks therefore see a smaller cache.
+
+    chunks: list of (Qw [Hq,w,dh], K [Hkv,len,dh], V [Hkv,len,dh]) widened inputs.
+    Returns (K_ret, V_ret [Hkv, B_last, dh], pos [Hkv, B_last] original token positions, history of per-step idx).
+    """
+    K_ret = V_ret = pos = None
+    seen = 0
+    hist = []
+    for c, (Qw, K, V) in enumerate(chunks):
+        Hkv, ln, _ = K.shape
+        new_pos = np.broadcast_to(np.arange(seen, seen + ln, dtype=np.int64), (Hkv, ln))
+        if K_ret is None:
+            Kc, Vc, pc = K, V, new_pos
+        else:
+            Kc = np.concatenate([K_ret, K], axis=1)
+            Vc = np.concatenate([V_ret, V], axis=1)
+            pc = np.concatenate([pos, new_pos], axis=1)
+        seen += ln
+        out = compress_layer(Qw, Kc, Vc, WO, kp=kp, budget_mode="uniform", budget=int(budgets[c]), alpha=alpha,
+                             eps=eps, scale=scale)
+        B = int(budgets[c])
+        idx = out["idx"].reshape(Hkv, B)
+        K_ret = np.stack([Kc[g][idx[g]] for g in range(Hkv)])
+        V_ret = np.stack([Vc[g][idx[g]] for g in range(Hkv)])
+        pos = np.stack([pc[g][idx[g]] for g in range(Hkv)])
+        hist.append(idx)
+    return K_ret, V_ret, pos, hist
+
+
 # ----------------------------------------------------------------------------
 # Diagnostics: the quantities of Section 3 (Definition 3.1, Theorems 3.2, 3.3,
 # 3.5, Assumption 3.4, relaxed bound).  Single query row, single head.

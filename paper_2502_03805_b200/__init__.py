@@ -5,4 +5,4 @@ Importing the package does not load the shared library; the first call does, and
 """
 from . import binding, build  # noqa: F401
 from .binding import *  # noqa: F401,F403
-from .session import CompressionSession, session_for, to_device, to_host  # noqa: F401,E402
+from .session import ChunkedPrefillCompressor, CompressionSession, session_for, to_device, to_host  # noqa: F401,E402

@@ -22,7 +22,7 @@ CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM, CKV_FLAG_PROTECT
 CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",
-           "criticalkv_select", "criticalkv_select_static", "criticalkv_compact", "criticalkv_compress",
+           "criticalkv_select", "criticalkv_select_static", "criticalkv_compact", "criticalkv_gather_positions", "criticalkv_compress",
            "criticalkv_host_staging_bytes", "criticalkv_compress_host", "criticalkv_selftest_bounded_wait", "criticalkv_device_status",
            "criticalkv_status_string", "criticalkv_last_cuda_error", "criticalkv_last_path",
            "criticalkv_launch_count")
@@ -66,6 +66,7 @@ def load():
     lib.criticalkv_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.criticalkv_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
     lib.criticalkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
+    lib.criticalkv_gather_positions.argtypes = [vp, dp, vp, vp, vp, vp, vp]
     lib.criticalkv_compress.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.criticalkv_host_staging_bytes.argtypes = [dp, C.POINTER(sz)]
     lib.criticalkv_compress_host.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -182,6 +183,12 @@ def criticalkv_compact(handle, desc, K, V, idx, offsets, K_out, V_out, stream=No
     rc = load().criticalkv_compact(handle, C.byref(desc), _ptr(K), _ptr(V), _ptr(idx), _ptr(offsets), _ptr(K_out),
                                    _ptr(V_out), _stream(stream))
     return _check(handle, rc, "criticalkv_compact", check)
+
+
+def criticalkv_gather_positions(handle, desc, pos_in, idx, offsets, pos_out, stream=None, check=True):
+    rc = load().criticalkv_gather_positions(handle, C.byref(desc), _ptr(pos_in), _ptr(idx), _ptr(offsets),
+                                            _ptr(pos_out), _stream(stream))
+    return _check(handle, rc, "criticalkv_gather_positions", check)
 
 
 def criticalkv_compress(handle, desc, Qw, K, V, WO, budgets_in, attn, vnorm, idx, offsets, stage, K_out, V_out, ws,

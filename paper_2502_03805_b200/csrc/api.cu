@@ -308,6 +308,25 @@ int criticalkv_compact(criticalkv_handle h, const criticalkv_desc* d, const void
   return record_cuda(h, e);
 }
 
+int criticalkv_gather_positions(criticalkv_handle h, const criticalkv_desc* d, const int32_t* pos_in,
+                                const int32_t* idx, const int32_t* offsets, int32_t* pos_out, void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (!pos_in || !idx || !offsets || !pos_out) return CKV_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(pos_in) | reinterpret_cast<uintptr_t>(idx) | reinterpret_cast<uintptr_t>(offsets) |
+       reinterpret_cast<uintptr_t>(pos_out)) & 3u)
+    return CKV_EALIGN;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  if (dd.btot == 0) return CKV_OK;
+  int launches = 0;
+  cudaError_t e = ckv::launch_gather_positions(dd, pos_in, idx, offsets, pos_out, (cudaStream_t)stream, &launches);
+  h->launches += launches;
+  return record_cuda(h, e);
+}
+
 int criticalkv_compress(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K, const void* V,
                         const void* WO, const int32_t* budgets_in, float* attn, float* vnorm, int32_t* idx,
                         int32_t* offsets, uint8_t* stage, void* K_out, void* V_out, void* ws, size_t ws_bytes,

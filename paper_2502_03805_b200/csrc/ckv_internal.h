@@ -66,4 +66,7 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
 cudaError_t launch_compact(const Dims& d, const void* K, const void* V, const int32_t* idx, const int32_t* offsets,
                            void* K_out, void* V_out, cudaStream_t st, int* launches);
 
+cudaError_t launch_gather_positions(const Dims& d, const int32_t* pos_in, const int32_t* idx, const int32_t* offsets,
+                                    int32_t* pos_out, cudaStream_t st, int* launches);
+
 }  // namespace ckv

@@ -46,7 +46,34 @@ __global__ void __launch_bounds__(kThreads) compact_kernel(CompactArgs p) {
   }
 }
 
+__global__ void gather_positions_kernel(const int32_t* __restrict__ pos_in, const int32_t* __restrict__ idx,
+                                        const int32_t* __restrict__ offsets, int32_t* __restrict__ pos_out, int Hkv,
+                                        int n, long long btot) {
+  __shared__ int32_t offs[65];
+  const int b = blockIdx.y;
+  for (int q = threadIdx.x; q <= Hkv; q += blockDim.x) offs[q] = offsets[(long long)b * (Hkv + 1) + q];
+  __syncthreads();
+  const long long total = min((long long)offs[Hkv], btot);
+  for (long long r = (long long)blockIdx.x * blockDim.x + threadIdx.x; r < total; r += (long long)gridDim.x * blockDim.x) {
+    int g = 0;
+    while (g + 1 < Hkv && r >= offs[g + 1]) ++g;
+    const int src = idx[(long long)b * btot + r];
+    if (src >= 0 && src < n) pos_out[(long long)b * btot + r] = pos_in[((long long)b * Hkv + g) * n + src];
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_gather_positions(const Dims& d, const int32_t* pos_in, const int32_t* idx, const int32_t* offsets,
+                                    int32_t* pos_out, cudaStream_t st, int* launches) {
+  long long ctas = (d.btot + 255) / 256;
+  if (ctas < 1) ctas = 1;
+  if (ctas > 148 * 8) ctas = 148 * 8;
+  dim3 grid((unsigned)ctas, d.nb);
+  gather_positions_kernel<<<grid, 256, 0, st>>>(pos_in, idx, offsets, pos_out, d.Hkv, d.n, d.btot);
+  *launches += 1;
+  return cudaGetLastError();
+}
 
 cudaError_t launch_compact(const Dims& d, const void* K, const void* V, const int32_t* idx, const int32_t* offsets,
                            void* K_out, void* V_out, cudaStream_t st, int* launches) {

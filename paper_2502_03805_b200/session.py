@@ -98,3 +98,40 @@ def session_for(wl, nb=1, **kw) -> CompressionSession:
     return CompressionSession(nb=nb, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp,
                               dtype=wl.dtype, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha,
                               eps=wl.eps, **kw)
+
+
+class ChunkedPrefillCompressor:
+    """Chunked prefill with eviction between chunks (uniform budgets): keeps the retained K, V and their original
+    token positions on the device; every step appends a chunk, calls criticalkv_compress on [retained ; chunk] and
+    keeps the rows the library selected.  Only buffer concatenation and reshaping happen here."""
+
+    def __init__(self, *, Hq, Hkv, dh, dm, w, pool_k, dtype, alpha=0.5, eps=1e-4, scale=0.0, flags=0, device=0):
+        self.kw = dict(Hq=Hq, Hkv=Hkv, dh=dh, dm=dm, w=w, pool_k=pool_k, dtype=dtype, alpha=alpha, eps=eps,
+                       scale=scale, flags=flags, device=device)
+        self.Hkv, self.dh = Hkv, dh
+        self.device = torch.device("cuda", device)
+        self.K = self.V = self.pos = None
+        self.seen = 0
+
+    def step(self, Qw, K_chunk, V_chunk, WO, budget):
+        """Qw [Hq,w,dh] (last w queries of the chunk), K_chunk, V_chunk [Hkv,len,dh], WO [Hq,dh,dm]: device tensors.
+        Compresses [retained ; chunk] to `budget` entries per KV head.  Returns the session used (its attn, vnorm,
+        idx are valid until the next step)."""
+        ln = K_chunk.shape[1]
+        new_pos = torch.arange(self.seen, self.seen + ln, dtype=torch.int32, device=self.device).expand(self.Hkv, ln)
+        if self.K is None:
+            Kc, Vc, pc = K_chunk.contiguous(), V_chunk.contiguous(), new_pos.contiguous()
+        else:
+            Kc = torch.cat([self.K, K_chunk], dim=1)
+            Vc = torch.cat([self.V, V_chunk], dim=1)
+            pc = torch.cat([self.pos, new_pos], dim=1).contiguous()
+        self.seen += ln
+        s = CompressionSession(nb=1, n=Kc.shape[1], budget_mode="uniform", budget=int(budget), want_stage=False,
+                               **self.kw)
+        s.compress(Qw, Kc, Vc, WO)
+        pos_out = torch.empty((1, max(s.btot, 1)), dtype=torch.int32, device=self.device)
+        B.criticalkv_gather_positions(s.handle, s.desc, pc, s.idx, s.offsets, pos_out)
+        self.K = s.K_out[0, : s.btot].reshape(self.Hkv, int(budget), self.dh)
+        self.V = s.V_out[0, : s.btot].reshape(self.Hkv, int(budget), self.dh)
+        self.pos = pos_out[0, : s.btot].reshape(self.Hkv, int(budget))
+        return s

@@ -518,6 +518,28 @@ def test_post_eviction_output_full_cache_is_plain_attention():
     np.testing.assert_allclose(one, np.repeat(V[4:5], w, axis=0), rtol=1e-12)
 
 
+def test_chunked_compress_single_chunk_and_positions():
+    from gen import make_layer, small_workload
+    wl = small_workload(n=120, w=8, kp=5, budget=30, cfg_id=71)
+    L = make_layer(wl)
+    # one chunk = plain compression; positions are the selected indices
+    K1, V1, pos, hist = oc.chunked_compress([(L.Qw, L.K, L.V)], L.WO, kp=wl.kp, w=wl.w, budgets=[30])
+    ref = oc.compress_layer(L.Qw, L.K, L.V, L.WO, kp=wl.kp, budget_mode="uniform", budget=30)
+    np.testing.assert_array_equal(pos.reshape(-1), ref["idx"])
+    np.testing.assert_array_equal(K1.reshape(-1, wl.dh), ref["K_hat"])
+    # two chunks: the second step sees [30 retained ; 60 new] and positions stay original, ascending, in range
+    L2 = make_layer(wl.with_(n=60), 1)
+    K2, V2, pos2, hist2 = oc.chunked_compress([(L.Qw, L.K, L.V), (L2.Qw, L2.K, L2.V)], L.WO, kp=wl.kp, w=wl.w,
+                                              budgets=[30, 40])
+    assert pos2.shape == (wl.Hkv, 40) and np.all(np.diff(pos2, axis=1) > 0) and pos2.max() < 180
+    for g in range(wl.Hkv):
+        old = pos2[g][pos2[g] < 120]
+        assert set(old.tolist()) <= set(pos[g].tolist())          # nothing evicted in step 1 comes back
+        for p, krow in zip(pos2[g], K2[g]):
+            src = L.K[g][p] if p < 120 else L2.K[g][p - 120]
+            np.testing.assert_array_equal(krow, src)
+
+
 def test_compress_layer_end_to_end_small():
     from gen import make_layer, small_workload
     wl = small_workload(n=96, w=8, kp=5, budget=20)

@@ -241,6 +241,31 @@ def test_adaptive_floor_and_protected_window_are_bit_exact_on_identical_scores(f
         assert list(np.diff(off)) == [budget // Hkv] * Hkv
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_chunked_prefill_matches_oracle(dtype):
+    # three prefill chunks with eviction after each: the retained positions and rows must match the oracle's
+    from paper_2502_03805_b200 import ChunkedPrefillCompressor, to_device, to_host
+    base = small_workload(cfg_id=180, dtype=dtype, Hq=4, Hkv=2, dh=128 if dtype == "bf16" else 64, dm=256, n=600,
+                          w=16, kp=5, budget=200)
+    lens, budgets = [600, 500, 300], [200, 300, 250]
+    Ls = [make_layer(base.with_(n=ln), c) for c, ln in enumerate(lens)]
+    WO = Ls[0].WO
+    Kr, Vr, pos, _ = oc.chunked_compress([(L.Qw, L.K, L.V) for L in Ls], WO, kp=base.kp, w=base.w, budgets=budgets)
+    cp = ChunkedPrefillCompressor(Hq=base.Hq, Hkv=base.Hkv, dh=base.dh, dm=base.dm, w=base.w, pool_k=base.kp,
+                                  dtype=dtype)
+    dWO = to_device(Ls[0].WO_store, dtype)
+    for L, b in zip(Ls, budgets):
+        cp.step(to_device(L.Qw_store, dtype), to_device(L.K_store, dtype), to_device(L.V_store, dtype), dWO, b)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(cp.pos.cpu().numpy(), pos)
+    from gen import bf16_bits_to_f32
+    Kg, Vg = to_host(cp.K), to_host(cp.V)
+    if dtype == "bf16":
+        Kg, Vg = bf16_bits_to_f32(Kg), bf16_bits_to_f32(Vg)
+    np.testing.assert_array_equal(Kg, Kr)
+    np.testing.assert_array_equal(Vg, Vr)
+
+
 def test_bounded_wait_times_out_and_reports_status():
     # a wait on a barrier nothing signals must end by itself, set CKV_ETIMEOUT, and leave the context usable
     import time
