@@ -43,6 +43,8 @@ def parse_args():
     p.add_argument("--impl", default="ours", choices=["ours", "reference"])
     p.add_argument("--cfg", type=int, default=3, help="workload id in gen.CONFIGS (3 = the headline 32-layer stack)")
     p.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
+    p.add_argument("--group-sum", action="store_true",
+                   help="measure the grouped-query shortcut of step 2 (CKV_FLAG_WO_GROUP_SUM) instead of the headline path")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     return p.parse_args()
@@ -189,7 +191,8 @@ def main():
     torch.cuda.synchronize()
     t_gen = time.time() - t_gen
 
-    s = session_for(wl, nb=nb, device=local, want_stage=False)
+    flags = B.CKV_FLAG_WO_GROUP_SUM if args.group_sum else 0
+    s = session_for(wl, nb=nb, device=local, want_stage=False, flags=flags)
     stream = torch.cuda.current_stream()
     gemm_ev = []
 
@@ -237,7 +240,7 @@ def main():
     # ---- end to end: host buffers, copies inside the timed region, layer by layer on two streams ----
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, wl, host, local, world)
+        e2e = run_e2e(args, wl, host, local, world, flags)
 
     ms_total = max_over_ranks(ms_total, dev)
     ms_per_step = ms_total / args.steps
@@ -245,7 +248,7 @@ def main():
 
     if rank == 0:
         peaks, how = load_peaks()
-        flops = 2.0 * wl.n * wl.dh * wl.dm * wl.Hq * nb
+        flops = 2.0 * wl.n * wl.dh * wl.dm * (wl.Hkv if args.group_sum else wl.Hq) * nb
         gemm_avg = sum(gemm_ms) / len(gemm_ms)
         achieved = flops / (gemm_avg * 1e-3) / 1e12
         peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
@@ -265,6 +268,7 @@ def main():
                 "config": {"workload": wl.name, "layers": nb, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.dh,
                            "d_model": wl.dm, "n": wl.n, "window": wl.w, "pool_kernel": wl.kp,
                            "budget": f"{wl.budget_mode} {wl.budget} per layer", "alpha": wl.alpha,
+                           "projection": "summed W_O slice per KV head" if args.group_sum else "per query head",
                            "l2": "inputs of one step (5.4 GB) exceed L2; layers are distinct buffers",
                            "ms_per_32_layer_compression": ms_per_step * 32.0 / nb},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
@@ -274,7 +278,7 @@ def main():
         dist.destroy_process_group()
 
 
-def run_e2e(args, wl, host, local, world):
+def run_e2e(args, wl, host, local, world, flags=0):
     """Same metric through criticalkv_compress_host: every step's inputs start in pinned host memory and its results
     (idx, offsets, compacted K and V) end there; the library streams the layers through two device staging buffers."""
     import torch
@@ -285,7 +289,7 @@ def run_e2e(args, wl, host, local, world):
     nb = wl.layers
     tdt = torch.bfloat16 if wl.dtype == "bf16" else torch.float32
     desc = B.make_desc(nb=nb, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp, dtype=wl.dtype,
-                       budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps)
+                       budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps, flags=flags)
     handle = B.criticalkv_create(local)
     staging = torch.empty(B.criticalkv_host_staging_bytes(desc), dtype=torch.uint8, device=dev)
     out_host = {"idx": torch.empty((nb, wl.btot), dtype=torch.int32).pin_memory(),
