@@ -435,6 +435,43 @@ def post_eviction_output(Qw_h, K_g, V_g, keep_idx, scale):
     return out
 
 
+DIAG_FIELDS = ("sigma", "mass_kept", "C", "C_stage1", "C_stage2", "nu_min", "L", "theta", "theta_hat",
+               "theta_relax")
+
+
+def row_diagnostics(Qw_h, K_g, V_g, WO_h, S1, S2, scale):
+    """Section 3 quantities of one query head for each of its w window rows and a given selection (S1, S2 = index
+    arrays of the two stages): per row j, with A = the row's causal softmax and nu = row L1 norms of V W^O,
+      sigma = sum_{S1} A (Assumption 3.4), mass_kept = sum_{S1+S2} A, C = sum_i A_i nu_i, C_stage1/2 = the same sum
+      over each stage, nu_min = min_i nu_i, L = || (A - A') V W^O ||_1 (Definition 3.1, A' by Theorem 3.2),
+      theta (Theorem 3.3), theta_hat (Theorem 3.5), theta_relax (relaxed bound of the appendix).
+    Returns [w, 10] float64 in the order of DIAG_FIELDS."""
+    Qw_h, K_g, V_g, WO_h = (np.asarray(x, dtype=F64) for x in (Qw_h, K_g, V_g, WO_h))
+    w, n = Qw_h.shape[0], K_g.shape[0]
+    A = window_softmax(Qw_h, K_g, scale)
+    Vp = V_g @ WO_h
+    nu = np.abs(Vp).sum(axis=1)
+    k1 = np.zeros(n, bool)
+    k1[np.asarray(S1, dtype=np.int64)] = True
+    k2 = np.zeros(n, bool)
+    k2[np.asarray(S2, dtype=np.int64)] = True
+    keep = k1 | k2
+    out = np.zeros((w, len(DIAG_FIELDS)), dtype=F64)
+    for j in range(w):
+        a = A[j]
+        sigma, mass = a[k1].sum(), a[keep].sum()
+        C, C1, C2 = (a * nu).sum(), (a[k1] * nu[k1]).sum(), (a[k2] * nu[k2]).sum()
+        a_kept = np.where(keep, a, 0.0) / mass if mass > 0 else np.zeros(n)
+        L = np.abs((a - a_kept) @ Vp).sum()
+        f_all = 2.0 - 1.0 / mass if mass > 0 else -np.inf
+        f_s1 = 2.0 - 1.0 / sigma if sigma > 0 else -np.inf
+        theta = C - f_all * (C1 + C2)
+        theta_hat = C - f_s1 * (C1 + C2)
+        theta_relax = C - f_s1 * C1 - nu.min() * f_s1 * a[k2].sum()
+        out[j] = (sigma, mass, C, C1, C2, nu.min(), L, theta, theta_hat, theta_relax)
+    return out
+
+
 def all_subsets(n, b):
     """Every subset of size b as a boolean mask (tiny n only)."""
     for comb in combinations(range(n), b):

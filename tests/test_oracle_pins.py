@@ -504,6 +504,37 @@ def test_attention_only_selection_minimises_relaxed_bound():
     assert set(min(vals, key=vals.get)) == set(S2.tolist())
 
 
+def test_row_diagnostics_agree_with_the_single_row_functions():
+    # the batched diagnostics restate theta / theta_hat / theta_relax / L: check them against the per-row functions
+    # that the brute-force theorem pins already cover, and against the masked softmax of Section 3.3
+    r = RNG(90)
+    n, w, dh, dm = 30, 4, 6, 9
+    Q, K = r.standard_normal((w, dh)), r.standard_normal((n, dh))
+    K[[3, 11, 20]] += 2.5 * Q[-1] / np.linalg.norm(Q[-1])
+    V, W = r.standard_normal((n, dh)) * np.exp(r.standard_normal((n, 1))), r.standard_normal((dh, dm))
+    sc = 1 / math.sqrt(dh)
+    S1, S2 = np.array([3, 11, 20, 25]), np.array([0, 7, 18])
+    D = oc.row_diagnostics(Q, K, V, W, S1, S2, sc)
+    A = oc.window_softmax(Q, K, sc)
+    Vp = V @ W
+    nu = np.abs(Vp).sum(axis=1)
+    k1 = np.isin(np.arange(n), S1)
+    k2 = np.isin(np.arange(n), S2)
+    for j in range(w):
+        vis = np.arange(n) <= n - w + j
+        logits = (Q[j] @ K.T) * sc
+        A_kept = oc.masked_softmax(np.where(vis, logits, -1e300), (k1 | k2) & vis)
+        f = dict(zip(oc.DIAG_FIELDS, D[j]))
+        assert abs(f["L"] - oc.perturbation(A[j], A_kept, Vp)) < 1e-10
+        assert abs(f["theta"] - oc.theta_bound(A[j], nu, k1 | k2)) < 1e-10
+        assert abs(f["theta_hat"] - oc.theta_hat_bound(A[j], nu, k1, k2)) < 1e-10
+        assert abs(f["theta_relax"] - oc.theta_relax_bound(A[j], nu, k1, k2)) < 1e-10
+        assert abs(f["sigma"] - A[j][k1].sum()) < 1e-14 and abs(f["nu_min"] - nu.min()) < 1e-14
+        assert f["L"] <= f["theta"] + 1e-12
+        if f["sigma"] > 0.5:
+            assert f["theta"] <= f["theta_hat"] + 1e-12 <= f["theta_relax"] + 2e-12
+
+
 def test_post_eviction_output_full_cache_is_plain_attention():
     r = RNG(16)
     n, w, dh = 20, 3, 4
