@@ -196,6 +196,22 @@ CKV_API int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc*
                                      size_t staging_bytes, void* stream);
 
 /*
+ * Perturbation diagnostics of Section 3 for a finished selection (not on the hot path).  For every query head and
+ * window row j, with A the causal softmax row of that query and nu = vnorm of the head:
+ *   diag[nb,Hq,w,10] = sigma (attention mass of the stage-1 set, Assumption 3.4), retained mass, C = sum_i A_i nu_i,
+ *   its parts over stage 1 and stage 2, min_i nu_i, L = ||(A - A') V W^O||_1 (Definition 3.1 with A' of Theorem 3.2),
+ *   theta (Theorem 3.3), theta_hat (Theorem 3.5), theta_relax (relaxed bound of the appendix).
+ * vnorm is the per-head output of criticalkv_score (not available with CKV_FLAG_WO_GROUP_SUM); idx, offsets and
+ * stage (required) come from criticalkv_select.  ws: criticalkv_diagnose_workspace_bytes, 256-byte aligned.
+ */
+#define CKV_DIAG_FIELDS 10
+CKV_API int criticalkv_diagnose_workspace_bytes(const criticalkv_desc* d, size_t* bytes);
+CKV_API int criticalkv_diagnose(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K,
+                                const void* V, const void* WO, const float* vnorm, const int32_t* idx,
+                                const int32_t* offsets, const uint8_t* stage, float* diag, void* ws, size_t ws_bytes,
+                                void* stream);
+
+/*
  * Self-test of the bounded device-side wait every tensor-core kernel uses: launches one CTA that waits, for at most
  * limit_ns nanoseconds, on a barrier nothing will ever signal.  The kernel must give up, write 0 to *observed_device
  * (a device int; 1 would mean the wait claimed success), set the status word to CKV_ETIMEOUT and end normally.

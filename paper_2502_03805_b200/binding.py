@@ -23,7 +23,8 @@ CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",
            "criticalkv_select", "criticalkv_select_static", "criticalkv_compact", "criticalkv_gather_positions", "criticalkv_compress",
-           "criticalkv_host_staging_bytes", "criticalkv_compress_host", "criticalkv_selftest_bounded_wait", "criticalkv_device_status",
+           "criticalkv_host_staging_bytes", "criticalkv_compress_host", "criticalkv_selftest_bounded_wait",
+           "criticalkv_diagnose_workspace_bytes", "criticalkv_diagnose", "criticalkv_device_status",
            "criticalkv_status_string", "criticalkv_last_cuda_error", "criticalkv_last_path",
            "criticalkv_launch_count")
 
@@ -70,6 +71,8 @@ def load():
     lib.criticalkv_compress.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.criticalkv_host_staging_bytes.argtypes = [dp, C.POINTER(sz)]
     lib.criticalkv_compress_host.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.criticalkv_diagnose_workspace_bytes.argtypes = [dp, C.POINTER(sz)]
+    lib.criticalkv_diagnose.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.criticalkv_selftest_bounded_wait.argtypes = [vp, C.c_uint64, vp, vp]
     lib.criticalkv_device_status.argtypes = [vp, vp, C.POINTER(i32)]
     lib.criticalkv_status_string.argtypes = [i32]
@@ -216,9 +219,29 @@ def criticalkv_compress_host(handle, desc, Qw, K, V, WO, budgets_in, idx, offset
     return _check(handle, rc, "criticalkv_compress_host", check)
 
 
+DIAG_FIELDS = ("sigma", "mass_kept", "C", "C_stage1", "C_stage2", "nu_min", "L", "theta", "theta_hat", "theta_relax")
+
+
+def criticalkv_diagnose_workspace_bytes(desc):
+    out = C.c_size_t()
+    rc = load().criticalkv_diagnose_workspace_bytes(C.byref(desc), C.byref(out))
+    if rc != CKV_OK:
+        raise CriticalKVError(rc, "criticalkv_diagnose_workspace_bytes")
+    return out.value
+
+
+def criticalkv_diagnose(handle, desc, Qw, K, V, WO, vnorm, idx, offsets, stage, diag, ws, ws_bytes=None, stream=None,
+                        check=True):
+    rc = load().criticalkv_diagnose(handle, C.byref(desc), _ptr(Qw), _ptr(K), _ptr(V), _ptr(WO), _ptr(vnorm),
+                                    _ptr(idx), _ptr(offsets), _ptr(stage), _ptr(diag), _ptr(ws),
+                                    _nbytes(ws, ws_bytes), _stream(stream))
+    return _check(handle, rc, "criticalkv_diagnose", check)
+
+
 def criticalkv_selftest_bounded_wait(handle, limit_ns, observed, stream=None, check=True):
     rc = load().criticalkv_selftest_bounded_wait(handle, int(limit_ns), _ptr(observed), _stream(stream))
-    return _check(handle, rc, "criticalkv_selftest_bounded_wait", check)
+    return _check(handle, rc, "criticalkv_selftest_bounded_wait",
+           "criticalkv_diagnose_workspace_bytes", "criticalkv_diagnose", check)
 
 
 def criticalkv_device_status(handle, stream=None):

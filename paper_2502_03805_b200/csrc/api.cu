@@ -480,6 +480,42 @@ int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc* d, cons
   return record_cuda(h, e);
 }
 
+int criticalkv_diagnose_workspace_bytes(const criticalkv_desc* d, size_t* bytes) {
+  if (!bytes) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  *bytes = score_layout(dd).total + align_up((size_t)dd.nb * dd.Hkv * dd.n, 256);
+  return CKV_OK;
+}
+
+int criticalkv_diagnose(criticalkv_handle h, const criticalkv_desc* d, const void* Qw, const void* K, const void* V,
+                        const void* WO, const float* vnorm, const int32_t* idx, const int32_t* offsets,
+                        const uint8_t* stage, float* diag, void* ws, size_t ws_bytes, void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (dd.group_sum) return CKV_ENOTSUP;  // the bounds are stated with per-head norms
+  if (!Qw || !K || !V || !WO || !vnorm || !idx || !offsets || !stage || !diag || !ws) return CKV_EINVAL;
+  if (!aligned16(Qw) || !aligned16(K) || !aligned16(V) || !aligned16(WO) || !aligned16(vnorm) || !aligned16(diag) ||
+      (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(offsets) & 3u) ||
+      (reinterpret_cast<uintptr_t>(ws) & 255u))
+    return CKV_EALIGN;
+  const ScoreLayout L = score_layout(dd);
+  if (ws_bytes < L.total + align_up((size_t)dd.nb * dd.Hkv * dd.n, 256)) return CKV_EWORKSPACE;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  char* base = (char*)ws;
+  ckv::ScoreWorkspace sw{(float*)(base + L.part_m), (float*)(base + L.part_l), (float*)(base + L.rowstat),
+                         (float*)(base + L.abar), (void*)(base + L.wsum)};
+  int launches = 0;
+  cudaError_t e = ckv::launch_diagnostics(dd, Qw, K, V, WO, vnorm, idx, offsets, stage, diag, sw,
+                                          (uint8_t*)(base + L.total), (cudaStream_t)stream, &launches);
+  h->launches += launches;
+  return record_cuda(h, e);
+}
+
 int criticalkv_selftest_bounded_wait(criticalkv_handle h, uint64_t limit_ns, int* observed_device, void* stream) {
   if (!h || !observed_device) return CKV_EINVAL;
   if (h->cc_major < 9) return CKV_ENOTSUP;

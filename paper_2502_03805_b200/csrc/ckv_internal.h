@@ -48,6 +48,12 @@ cudaError_t launch_vnorm_simt(const Dims& d, const void* V, const void* WO, floa
 cudaError_t launch_attn_combine(const float* part_m, const float* part_l, float* rowstat, int rows, int nchunks,
                                 int w, cudaStream_t st);
 cudaError_t launch_maxpool(const float* abar, float* attn, int n, int kp, int nrows, cudaStream_t st);
+cudaError_t launch_window_stats_simt(const Dims& d, const void* Qw, const void* K, const ScoreWorkspace& ws,
+                                     cudaStream_t st, int* launches);
+cudaError_t launch_diagnostics(const Dims& d, const void* Qw, const void* K, const void* V, const void* WO,
+                               const float* vnorm, const int32_t* idx, const int32_t* offsets, const uint8_t* stage,
+                               float* diag, const ScoreWorkspace& ws, uint8_t* stage_of, cudaStream_t st,
+                               int* launches);
 // Tensor-core window attention (bf16).  cudaErrorNotSupported = shape or layout outside what it handles.
 cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K, float* attn,
                                     const ScoreWorkspace& ws, int sm_count, int* status_word, cudaStream_t st,

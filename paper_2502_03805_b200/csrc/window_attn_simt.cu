@@ -13,38 +13,11 @@
 #include <math.h>
 
 #include "ckv_internal.h"
+#include "simt_common.cuh"
 
 namespace ckv {
 namespace {
 
-constexpr int kThreads = kAttnChunk;  // one key per thread
-
-template <typename T>
-struct Vec16;  // 16-byte global load, widened to float
-template <>
-struct Vec16<float> {
-  static constexpr int kElems = 4;
-  __device__ static void load(const float* p, float* out) {
-    float4 v = *reinterpret_cast<const float4*>(p);
-    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
-  }
-};
-template <>
-struct Vec16<__nv_bfloat16> {
-  static constexpr int kElems = 8;
-  __device__ static void load(const __nv_bfloat16* p, float* out) {
-    uint4 v = *reinterpret_cast<const uint4*>(p);
-    const uint32_t u[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      out[2 * i] = __uint_as_float(u[i] << 16);
-      out[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
-    }
-  }
-};
-
-__device__ __forceinline__ float to_float(float x) { return x; }
-__device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
 
 struct AttnArgs {
   const void* Qw;
@@ -57,31 +30,6 @@ struct AttnArgs {
   float scale;
   long long qs[3], ks[3];
 };
-
-// Logits of window rows 0..WT-1 for this thread's key; rows >= w come out as 0 (their queries are zero-filled).
-template <typename T, int DH, int WT>
-__device__ __forceinline__ void key_logits(const T* krow, const float* q_s, float (&acc)[WT]) {
-#pragma unroll
-  for (int j = 0; j < WT; ++j) acc[j] = 0.f;
-  constexpr int E = Vec16<T>::kElems;
-#pragma unroll 1
-  for (int t = 0; t < DH; t += E) {
-    float kf[E];
-    Vec16<T>::load(krow + t, kf);
-#pragma unroll
-    for (int j = 0; j < WT; ++j) {
-      const float4* qv = reinterpret_cast<const float4*>(q_s + j * DH + t);
-#pragma unroll
-      for (int e4 = 0; e4 < E / 4; ++e4) {
-        float4 q = qv[e4];
-        acc[j] = fmaf(q.x, kf[4 * e4 + 0], acc[j]);
-        acc[j] = fmaf(q.y, kf[4 * e4 + 1], acc[j]);
-        acc[j] = fmaf(q.z, kf[4 * e4 + 2], acc[j]);
-        acc[j] = fmaf(q.w, kf[4 * e4 + 3], acc[j]);
-      }
-    }
-  }
-}
 
 template <typename T, int DH, int WT>
 __device__ __forceinline__ void stage_queries(const AttnArgs& a, int b, int h, float* q_s) {
@@ -219,6 +167,28 @@ cudaError_t run(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, 
   return cudaGetLastError();
 }
 
+// Only the row statistics (max, 1 / (w * sum)) of every window row: first pass and merge.
+template <typename T, int DH, int WT>
+cudaError_t run_stats(const Dims& d, const AttnArgs& a, cudaStream_t st, int* launches) {
+  const size_t smem = (size_t)(WT * DH + (kThreads / 32) * WT + 2 * WT) * sizeof(float);
+  auto k1 = attn_pass_kernel<T, DH, WT, false>;
+  cudaError_t e = cudaFuncSetAttribute(k1, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  dim3 grid(a.nchunks, d.Hq, d.nb);
+  k1<<<grid, kThreads, smem, st>>>(a);
+  const int rows = d.nb * d.Hq * d.w;
+  attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
+  *launches += 2;
+  return cudaGetLastError();
+}
+
+template <typename T, int DH>
+cudaError_t run_stats_w(const Dims& d, const AttnArgs& a, cudaStream_t st, int* launches) {
+  if (d.w <= 16) return run_stats<T, DH, 16>(d, a, st, launches);
+  if (d.w <= 32) return run_stats<T, DH, 32>(d, a, st, launches);
+  return run_stats<T, DH, 64>(d, a, st, launches);
+}
+
 template <typename T, int DH>
 cudaError_t run_w(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, int* launches) {
   if (d.w <= 16) return run<T, DH, 16>(d, a, attn, st, launches);
@@ -238,6 +208,26 @@ cudaError_t launch_maxpool(const float* abar, float* attn, int n, int kp, int nr
   dim3 pgrid((n + 255) / 256, nrows);
   maxpool_kernel<<<pgrid, 256, 0, st>>>(abar, attn, n, kp);
   return cudaGetLastError();
+}
+
+static AttnArgs make_attn_args(const Dims& d, const void* Qw, const void* K, const ScoreWorkspace& ws) {
+  AttnArgs a;
+  a.Qw = Qw; a.K = K;
+  a.part_m = ws.part_m; a.part_l = ws.part_l; a.rowstat = ws.rowstat; a.abar = ws.abar;
+  a.Hq = d.Hq; a.G = d.G; a.n = d.n; a.w = d.w;
+  a.nchunks = (d.n + kAttnChunk - 1) / kAttnChunk;
+  a.scale = d.scale;
+  for (int i = 0; i < 3; ++i) { a.qs[i] = d.qs[i]; a.ks[i] = d.ks[i]; }
+  return a;
+}
+
+cudaError_t launch_window_stats_simt(const Dims& d, const void* Qw, const void* K, const ScoreWorkspace& ws,
+                                     cudaStream_t st, int* launches) {
+  const AttnArgs a = make_attn_args(d, Qw, K, ws);
+  if (d.dtype == CKV_F32)
+    return d.dh == 64 ? run_stats_w<float, 64>(d, a, st, launches) : run_stats_w<float, 128>(d, a, st, launches);
+  return d.dh == 64 ? run_stats_w<__nv_bfloat16, 64>(d, a, st, launches)
+                    : run_stats_w<__nv_bfloat16, 128>(d, a, st, launches);
 }
 
 cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K, float* attn,

@@ -266,6 +266,37 @@ def test_chunked_prefill_matches_oracle(dtype):
     np.testing.assert_array_equal(Vg, Vr)
 
 
+@pytest.mark.parametrize("kw", [
+    dict(dtype="f32", n=500, w=16, kp=5, budget=120, dh=64, dm=192, Hq=4, Hkv=2),
+    dict(dtype="bf16", n=1100, w=32, kp=7, budget=300, dh=128, dm=256, Hq=4, Hkv=2),
+    dict(dtype="bf16", n=700, w=64, kp=7, budget_mode="adaptive", budget=500, dh=128, dm=128, Hq=6, Hkv=2),
+])
+def test_perturbation_diagnostics_match_oracle(kw):
+    # sigma, L, theta, theta_hat, theta_relax of Section 3 for the GPU's own selection, against the oracle's formulas
+    from paper_2502_03805_b200 import binding as B, session_for, to_device
+    wl = small_workload(cfg_id=190, **kw)
+    L = make_layer(wl, 0)
+    s = session_for(wl, nb=1)
+    Q, K, V, WO = (to_device(getattr(L, k)[None], wl.dtype) for k in ("Qw_store", "K_store", "V_store", "WO_store"))
+    s.compress(Q, K, V, WO)
+    diag = torch.zeros((1, wl.Hq, wl.w, 10), dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.criticalkv_diagnose_workspace_bytes(s.desc), dtype=torch.uint8, device="cuda")
+    B.criticalkv_diagnose(s.handle, s.desc, Q, K, V, WO, s.vnorm, s.idx, s.offsets, s.stage, diag, ws)
+    torch.cuda.synchronize()
+    assert s.device_status() == 0
+    got = diag[0].cpu().numpy().astype(np.float64)
+    idx, off, st = s.idx[0].cpu().numpy(), s.offsets[0].cpu().numpy(), s.stage[0].cpu().numpy()
+    for h in range(wl.Hq):
+        g = h // wl.G
+        seg, sst = idx[off[g]:off[g + 1]], st[off[g]:off[g + 1]]
+        ref = oc.row_diagnostics(L.Qw[h], L.K[g], L.V[g], L.WO[h], seg[sst == 1], seg[sst == 2], wl.scale)
+        C = ref[:, 2:3]
+        # sums of n float32 terms; the bounds subtract nearly equal quantities, so compare relative to C
+        np.testing.assert_allclose(got[h][:, :6], ref[:, :6], rtol=2e-3, atol=1e-6)
+        assert np.all(np.abs(got[h][:, 6:] - ref[:, 6:]) <= 2e-3 * C + 1e-6), (h, got[h][:, 6:], ref[:, 6:])
+        assert np.all(got[h][:, 6] <= got[h][:, 7] * (1 + 1e-3) + 1e-6)          # L <= theta (Theorem 3.3)
+
+
 def test_bounded_wait_times_out_and_reports_status():
     # a wait on a barrier nothing signals must end by itself, set CKV_ETIMEOUT, and leave the context usable
     import time
