@@ -62,7 +62,9 @@ typedef enum {
 
 typedef enum { CKV_F32 = 0, CKV_BF16 = 1 } criticalkv_dtype;
 typedef enum { CKV_BUDGET_UNIFORM = 0, CKV_BUDGET_FLAT_ADAPTIVE = 1, CKV_BUDGET_GIVEN = 2 } criticalkv_budget_mode;
-typedef enum { CKV_NORM_L1 = 0 } criticalkv_norm;
+/* CKV_NORM_L1: the paper's method.  CKV_NORM_L2: vnorm = ||V W^O_h||_2 (appendix on the distance metric), computed
+   through the Gram matrix W^O_h W^O_h^T, d_model / head_dim times fewer flops than the L1 projection. */
+typedef enum { CKV_NORM_L1 = 0, CKV_NORM_L2 = 1 } criticalkv_norm;
 
 enum {
   CKV_FLAG_WO_SHARED = 1u << 0,   /* WO has no nb dimension (one projection for the whole call)             */

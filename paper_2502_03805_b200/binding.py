@@ -17,7 +17,7 @@ _lib = None
 CKV_OK, CKV_EINVAL, CKV_ENOTSUP, CKV_EALIGN, CKV_EWORKSPACE, CKV_ECUDA, CKV_ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 CKV_F32, CKV_BF16 = 0, 1
 CKV_BUDGET_UNIFORM, CKV_BUDGET_FLAT_ADAPTIVE, CKV_BUDGET_GIVEN = 0, 1, 2
-CKV_NORM_L1 = 0
+CKV_NORM_L1, CKV_NORM_L2 = 0, 1
 CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM, CKV_FLAG_PROTECT_WINDOW = 1, 2, 4, 8
 CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 

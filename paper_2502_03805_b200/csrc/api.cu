@@ -51,7 +51,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (d->dtype != CKV_F32 && d->dtype != CKV_BF16) return CKV_EINVAL;
   if (!(d->alpha >= 0.f && d->alpha <= 1.f)) return CKV_EINVAL;
   if (!(d->eps >= 0.f) || !isfinite(d->eps)) return CKV_EINVAL;
-  if (d->norm != CKV_NORM_L1) return CKV_ENOTSUP;
+  if (d->norm != CKV_NORM_L1 && d->norm != CKV_NORM_L2) return CKV_EINVAL;
   if (d->reserved != 0 || d->reserved2 != 0) return CKV_EINVAL;
   if (!(d->adaptive_floor >= 0.f && d->adaptive_floor <= 1.f)) return CKV_EINVAL;
   if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM |
@@ -80,6 +80,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   o->wo_shared = (d->flags & CKV_FLAG_WO_SHARED) ? 1 : 0;
   o->group_sum = (d->flags & CKV_FLAG_WO_GROUP_SUM) ? 1 : 0;
   o->protect_window = (d->flags & CKV_FLAG_PROTECT_WINDOW) ? 1 : 0;
+  o->norm = d->norm;
   o->floor_b = 0;
   if (d->budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
     long long fb = (long long)floor((double)d->adaptive_floor * (double)d->budget / (double)d->Hkv);
@@ -101,7 +102,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
 }
 
 struct ScoreLayout {
-  size_t part_m, part_l, rowstat, abar, wsum, total;
+  size_t part_m, part_l, rowstat, abar, wsum, gram, total;
 };
 ScoreLayout score_layout(const Dims& d) {
   ScoreLayout L;
@@ -117,6 +118,8 @@ ScoreLayout score_layout(const Dims& d) {
   L.wsum = off;
   if (d.group_sum)
     off = align_up(off + (size_t)(d.wo_shared ? 1 : d.nb) * d.Hkv * d.dh * d.dm * (d.dtype == CKV_F32 ? 4 : 2), 256);
+  L.gram = off;
+  if (d.norm == CKV_NORM_L2) off = align_up(off + ckv::vnorm_l2_workspace_bytes(d), 1024);
   L.total = off;
   return L;
 }
@@ -216,7 +219,7 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
   cudaStream_t st = (cudaStream_t)stream;
   char* base = (char*)ws;
   ckv::ScoreWorkspace sw{(float*)(base + L.part_m), (float*)(base + L.part_l), (float*)(base + L.rowstat),
-                         (float*)(base + L.abar), (void*)(base + L.wsum)};
+                         (float*)(base + L.abar), (void*)(base + L.wsum), (void*)(base + L.gram)};
   int launches = 0, path = 0;
   cudaError_t e = cudaSuccess;
   if (attn) {
@@ -242,7 +245,12 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
     dd.Hq = dd.Hkv;
     dd.G = 1;
   }
-  if (e == cudaSuccess && vnorm) {
+  if (e == cudaSuccess && vnorm && dd.norm == CKV_NORM_L2) {
+    int tc = 0;
+    e = ckv::launch_vnorm_l2(dd, V, WO, vnorm, sw.gram, h->sm_count, h->cc_major,
+                             (d->flags & CKV_FLAG_FORCE_SIMT) != 0, h->status_word, st, &launches, &tc);
+    path |= tc ? 2 : 8;
+  } else if (e == cudaSuccess && vnorm) {
     bool done = false;
     if (dd.dtype == CKV_BF16 && !(d->flags & CKV_FLAG_FORCE_SIMT) && h->cc_major == 10) {
       e = ckv::launch_vnorm_umma(dd, V, WO, vnorm, h->sm_count, h->status_word, st, &launches);
@@ -508,7 +516,7 @@ int criticalkv_diagnose(criticalkv_handle h, const criticalkv_desc* d, const voi
   if (!guard.ok) return CKV_ECUDA;
   char* base = (char*)ws;
   ckv::ScoreWorkspace sw{(float*)(base + L.part_m), (float*)(base + L.part_l), (float*)(base + L.rowstat),
-                         (float*)(base + L.abar), (void*)(base + L.wsum)};
+                         (float*)(base + L.abar), (void*)(base + L.wsum), (void*)(base + L.gram)};
   int launches = 0;
   cudaError_t e = ckv::launch_diagnostics(dd, Qw, K, V, WO, vnorm, idx, offsets, stage, diag, sw,
                                           (uint8_t*)(base + L.total), (cudaStream_t)stream, &launches);

@@ -18,6 +18,7 @@ struct Dims {
   int wo_shared;
   int group_sum;      // CKV_FLAG_WO_GROUP_SUM
   int protect_window; // CKV_FLAG_PROTECT_WINDOW
+  int norm;           // criticalkv_norm
   long long floor_b;  // guaranteed entries per KV head (adaptive budgets)
   long long qs[3], ks[3], vs[3];  // element strides: nb, head, row
 };
@@ -31,6 +32,7 @@ struct ScoreWorkspace {   // carved out of the caller's workspace by the API lay
   float* rowstat;   // [nb*Hq*w, 2]         final (max, 1/(w*sum))
   float* abar;      // [nb*Hq, n]           window-mean attention before pooling
   void* wsum;       // [nbw, Hkv, dh, dm]   group-summed W^O (CKV_FLAG_WO_GROUP_SUM only)
+  void* gram;       // [nbw, Hq, dh, dh]    W^O_h W^O_h^T (CKV_NORM_L2 only): float32, or bf16 hi and lo parts
 };
 
 struct SelectWorkspace {
@@ -66,6 +68,11 @@ cudaError_t launch_bounded_wait_selftest(int* status_word, unsigned long long li
                                          cudaStream_t st);
 // W_tilde[bw, g] = round(sum_h WO[bw, g*G + h]) for the group-summed projection variant.
 cudaError_t launch_wo_group_sum(const Dims& d, const void* WO, void* wsum, cudaStream_t st, int* launches);
+// L2 variant of step 2 through the Gram matrix.
+size_t vnorm_l2_workspace_bytes(const Dims& d);
+cudaError_t launch_vnorm_l2(const Dims& d, const void* V, const void* WO, float* vnorm, void* gram, int sm_count,
+                            int cc_major, bool force_simt, int* status_word, cudaStream_t st, int* launches,
+                            int* used_tensor_cores);
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word);

@@ -31,12 +31,12 @@ class CompressionSession:
     """Holds a handle, a descriptor and the device buffers of one problem shape."""
 
     def __init__(self, *, nb, Hq, Hkv, dh, dm, n, w, pool_k, dtype, budget_mode, budget, alpha=0.5, eps=1e-4,
-                 scale=0.0, flags=0, device=0, want_stage=True, adaptive_floor=0.0):
+                 scale=0.0, flags=0, device=0, want_stage=True, adaptive_floor=0.0, norm=0):
         self.device = torch.device("cuda", device)
         self.dtype = dtype
         self.desc = B.make_desc(nb=nb, Hq=Hq, Hkv=Hkv, dh=dh, dm=dm, n=n, w=w, pool_k=pool_k, dtype=dtype,
                                 budget_mode=budget_mode, budget=budget, alpha=alpha, eps=eps, scale=scale,
-                                flags=flags, adaptive_floor=adaptive_floor)
+                                flags=flags, adaptive_floor=adaptive_floor, norm=norm)
         self.handle = B.criticalkv_create(device)
         self.btot = budget * Hkv if budget_mode == "uniform" else budget
         sb, tb = B.criticalkv_workspace_bytes(self.desc)

@@ -128,21 +128,22 @@ def assert_post_eviction_output(L, wl, ref_sel, gpu_idx, gpu_offsets, heads=None
     return worst
 
 
-def oracle_layer(L, wl, *, nu=None, P=None, group_sum=False):
+def oracle_layer(L, wl, *, nu=None, P=None, group_sum=False, norm="l1"):
     """Oracle scores and selection of one generated layer."""
     if P is None:
         P = oc.pooled_window_attention(L.Qw, L.K, wl.kp, wl.scale)
     if nu is None:
-        nu = oc.projection_norm_group_sum(L.V, L.WO, wl.G, wl.dtype) if group_sum else oc.projection_norm(L.V, L.WO)
+        nu = (oc.projection_norm_group_sum(L.V, L.WO, wl.G, wl.dtype, norm=norm) if group_sum
+              else oc.projection_norm(L.V, L.WO, norm=norm))
     sel = oc.select(P, nu, G=wl.G, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps,
                     group_sum=group_sum)
     return P, nu, sel
 
 
-def check_layer_against_oracle(L, wl, out, *, full_output_check=True, group_sum=False):
+def check_layer_against_oracle(L, wl, out, *, full_output_check=True, group_sum=False, norm="l1"):
     """out: dict of host arrays attn, vnorm [Hq,n] ([Hkv,n] for the group-summed variant); idx, stage [Btot];
     offsets [Hkv+1]; K_out, V_out [Btot, dh].  Returns a report with the worst errors."""
-    P, nu, sel = oracle_layer(L, wl, group_sum=group_sum)
+    P, nu, sel = oracle_layer(L, wl, group_sum=group_sum, norm=norm)
     rep = dict(attn_err=assert_scores_close(out["attn"], P, "attn"),
                vnorm_err=assert_scores_close(out["vnorm"], nu, "vnorm"))
     rep.update(compare_selection(sel, out["idx"], out["offsets"], out.get("stage"), n=wl.n, alpha=wl.alpha,

@@ -297,6 +297,31 @@ def test_perturbation_diagnostics_match_oracle(kw):
         assert np.all(got[h][:, 6] <= got[h][:, 7] * (1 + 1e-3) + 1e-6)          # L <= theta (Theorem 3.3)
 
 
+@pytest.mark.parametrize("kw,tensor_cores", [
+    (dict(dtype="bf16", n=1300, w=32, kp=7, budget=180, dh=128, dm=512, Hq=8, Hkv=2), True),
+    (dict(dtype="bf16", n=4500, w=32, kp=7, budget_mode="adaptive", budget=2000, dh=128, dm=1096, Hq=12, Hkv=4), True),
+    (dict(dtype="f32", n=500, w=16, kp=5, budget=70, dh=64, dm=192, Hq=6, Hkv=2), False),
+    (dict(dtype="bf16", n=900, w=16, kp=5, budget=100, dh=64, dm=256, Hq=4, Hkv=2), False),
+])
+def test_l2_norm_variant(kw, tensor_cores):
+    # CKV_NORM_L2: ||V W^O_h||_2 through the Gram matrix, against the oracle's materialised product
+    from paper_2502_03805_b200 import binding as B, session_for, to_device, to_host
+    wl = small_workload(cfg_id=200, **kw)
+    Ls = [make_layer(wl, l) for l in range(2)]
+    s = session_for(wl, nb=2, norm=B.CKV_NORM_L2)
+    Q, K, V, WO = (to_device(np.stack([getattr(L, k) for L in Ls]), wl.dtype)
+                   for k in ("Qw_store", "K_store", "V_store", "WO_store"))
+    s.compress(Q, K, V, WO)
+    torch.cuda.synchronize()
+    assert s.device_status() == 0
+    assert bool(s.last_path & 2) == tensor_cores
+    for b, L in enumerate(Ls):
+        out = dict(attn=to_host(s.attn[b]), vnorm=to_host(s.vnorm[b]), idx=to_host(s.idx[b]),
+                   offsets=to_host(s.offsets[b]), stage=to_host(s.stage[b]), K_out=to_host(s.K_out[b]),
+                   V_out=to_host(s.V_out[b]))
+        pu.check_layer_against_oracle(L, wl, out, norm="l2")
+
+
 def test_bounded_wait_times_out_and_reports_status():
     # a wait on a barrier nothing signals must end by itself, set CKV_ETIMEOUT, and leave the context usable
     import time
