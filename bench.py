@@ -45,6 +45,7 @@ def parse_args():
     p.add_argument("--layers", type=int, default=0, help="override the number of layers (debugging)")
     p.add_argument("--group-sum", action="store_true",
                    help="measure the grouped-query shortcut of step 2 (CKV_FLAG_WO_GROUP_SUM) instead of the headline path")
+    p.add_argument("--l2", action="store_true", help="measure the L2-norm variant of step 2 (CKV_NORM_L2, Gram matrix)")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     return p.parse_args()
@@ -192,7 +193,7 @@ def main():
     t_gen = time.time() - t_gen
 
     flags = B.CKV_FLAG_WO_GROUP_SUM if args.group_sum else 0
-    s = session_for(wl, nb=nb, device=local, want_stage=False, flags=flags)
+    s = session_for(wl, nb=nb, device=local, want_stage=False, flags=flags, norm=1 if args.l2 else 0)
     stream = torch.cuda.current_stream()
     gemm_ev = []
 
@@ -248,7 +249,10 @@ def main():
 
     if rank == 0:
         peaks, how = load_peaks()
-        flops = 2.0 * wl.n * wl.dh * wl.dm * (wl.Hkv if args.group_sum else wl.Hq) * nb
+        heads = wl.Hkv if args.group_sum else wl.Hq
+        flops = 2.0 * wl.n * wl.dh * wl.dm * heads * nb
+        if args.l2:   # Gram matrix + two-part quadratic form
+            flops = (2.0 * wl.dh * wl.dh * wl.dm + 2.0 * 2.0 * wl.n * wl.dh * wl.dh) * heads * nb
         gemm_avg = sum(gemm_ms) / len(gemm_ms)
         achieved = flops / (gemm_avg * 1e-3) / 1e12
         peak = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
@@ -268,7 +272,8 @@ def main():
                 "config": {"workload": wl.name, "layers": nb, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.dh,
                            "d_model": wl.dm, "n": wl.n, "window": wl.w, "pool_kernel": wl.kp,
                            "budget": f"{wl.budget_mode} {wl.budget} per layer", "alpha": wl.alpha,
-                           "projection": "summed W_O slice per KV head" if args.group_sum else "per query head",
+                           "projection": ("summed W_O slice per KV head" if args.group_sum else "per query head") +
+                                         (", L2 norm via Gram matrix" if args.l2 else ", L1 norm"),
                            "l2": "inputs of one step (5.4 GB) exceed L2; layers are distinct buffers",
                            "ms_per_32_layer_compression": ms_per_step * 32.0 / nb},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
