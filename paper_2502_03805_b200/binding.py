@@ -240,8 +240,7 @@ def criticalkv_diagnose(handle, desc, Qw, K, V, WO, vnorm, idx, offsets, stage, 
 
 def criticalkv_selftest_bounded_wait(handle, limit_ns, observed, stream=None, check=True):
     rc = load().criticalkv_selftest_bounded_wait(handle, int(limit_ns), _ptr(observed), _stream(stream))
-    return _check(handle, rc, "criticalkv_selftest_bounded_wait",
-           "criticalkv_diagnose_workspace_bytes", "criticalkv_diagnose", check)
+    return _check(handle, rc, "criticalkv_selftest_bounded_wait", check)
 
 
 def criticalkv_device_status(handle, stream=None):
