@@ -261,6 +261,14 @@ def main():
                     "peak_source": f"{how} (sustained bf16, kernel timed inside a long step)",
                     "ms_per_launch": gemm_avg, "flops_per_launch": flops, "traffic": None,
                     "tensor_core_path": bool(path & 2)}
+        if args.cfg == 3 and not args.group_sum and not args.l2 and (path & 2):
+            # dram__bytes_read.sum + dram__bytes_write.sum of vnorm_umma_kernel<128> from the ncu capture summarised in
+            # profiles/vnorm_umma_cfg3.md: 211.66 MB for 2 layers; every layer touches its own V, W_O and output once,
+            # so the traffic of a launch is proportional to the layers it processes
+            roofline["traffic"] = 211.66e6 / 2 * nb
+            roofline["traffic_unit"] = "bytes per launch (ncu, 2-layer capture scaled by layers)"
+            roofline["algorithmic_bytes"] = (2.0 * wl.Hkv * wl.n * wl.dh + 2.0 * wl.Hq * wl.dh * wl.dm +
+                                             4.0 * wl.Hq * wl.n) * nb
         cpu = None
         if not args.no_cpu_baseline:
             entries, dt, cores = oracle_sample(wl, 0)
