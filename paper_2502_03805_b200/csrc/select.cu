@@ -9,6 +9,8 @@
 //
 // Top-k is a radix *select* (4 passes of 8 bits over order-preserving integer keys) followed by an ordered walk that
 // resolves ties by index and compacts with warp ballots: no sort, no floating-point atomics, bit-reproducible.
+#include <cooperative_groups.h>
+
 #include "ckv_internal.h"
 
 namespace ckv {
@@ -278,6 +280,120 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_kernel(const floa
   }
 }
 
+// The same allocation spread over a thread-block cluster: CTA r of the cluster owns Hkv / cluster_size whole KV heads of
+// one nb slice, builds the digit histogram of its share, and every CTA sums the histograms of all ranks through
+// distributed shared memory, so all of them walk the same radix-select decisions without any broadcast.  Two hardware
+// cluster barriers per pass (histograms complete / histograms consumed).  Rank 0 finally reads every rank's per-head
+// counts and hands out the ties in flattened (g, i) order.
+struct ClusterShared {
+  uint32_t hist[kSelWarps][256];
+  uint32_t total[256];    // this CTA's histogram of the current pass (read by the peers)
+  uint32_t gtotal[256];   // sum over the cluster
+  uint32_t cnt_gt[64], cnt_eq[64];
+  uint32_t prefix, krem;
+};
+
+__global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(const float* __restrict__ a,
+                                                                              int32_t* __restrict__ budgets, int Hkv,
+                                                                              int n, long long btotal, int floor_b) {
+  namespace cg = cooperative_groups;
+  cg::cluster_group cluster = cg::this_cluster();
+  __shared__ ClusterShared sh;
+  const int cs = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
+  const int b = blockIdx.x / cs;
+  const int heads = Hkv / cs, g0 = rank * heads;
+  const float* ab = a + (long long)b * Hkv * n;
+  int32_t* out = budgets + (long long)b * Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (btotal <= 0) {   // uniform across the cluster: nobody reaches a cluster barrier
+    if (tid < heads) out[g0 + tid] = min(floor_b, n);
+    return;
+  }
+  const long long count = (long long)heads * n;
+  const float* mine = ab + (long long)g0 * n;
+  if (tid == 0) { sh.prefix = 0; sh.krem = (uint32_t)btotal; }
+  uint32_t known = 0;
+  for (int pass = 0; pass < 4; ++pass) {
+    const int shift = 24 - 8 * pass;
+    for (int e = tid; e < kSelWarps * 256; e += kSelThreads) (&sh.hist[0][0])[e] = 0;
+    __syncthreads();
+    const uint32_t prefix = sh.prefix;
+    for (long long i = tid; i < count; i += kSelThreads) {
+      const uint32_t key = order_key(mine[i]);
+      if ((key & known) == prefix) atomicAdd(&sh.hist[warp][(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 256) {
+      uint32_t s = 0;
+      for (int wq = 0; wq < kSelWarps; ++wq) s += sh.hist[wq][tid];
+      sh.total[tid] = s;
+    }
+    cluster.sync();   // every rank's total[] is complete
+    if (tid < 256) {
+      uint32_t s = 0;
+      for (int q = 0; q < cs; ++q) s += cluster.map_shared_rank(sh.total, q)[tid];
+      sh.gtotal[tid] = s;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      uint32_t m = 0;
+      for (int q = 0; q < 8; ++q) m += sh.gtotal[lane * 8 + q];
+      uint32_t above = m;
+      for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t v = __shfl_down_sync(0xffffffffu, above, o);
+        if (lane + o < 32) above += v;
+      }
+      above -= m;
+      const uint32_t krem = sh.krem;
+      if (above < krem && krem <= above + m) {
+        uint32_t acc = above;
+        for (int q = 7; q >= 0; --q) {
+          const uint32_t cnt = sh.gtotal[lane * 8 + q];
+          if (acc + cnt >= krem) {
+            sh.prefix = prefix | ((uint32_t)(lane * 8 + q) << shift);
+            sh.krem = krem - acc;
+            break;
+          }
+          acc += cnt;
+        }
+      }
+    }
+    known |= 0xffu << shift;
+    cluster.sync();   // peers are done reading total[] before the next pass rewrites it
+  }
+  const uint32_t T = sh.prefix, r = sh.krem;
+  if (tid < 64) { sh.cnt_gt[tid] = 0; sh.cnt_eq[tid] = 0; }
+  __syncthreads();
+  for (int g = 0; g < heads; ++g) {
+    uint32_t gt = 0, eq = 0;
+    for (int i = tid; i < n; i += kSelThreads) {
+      const uint32_t key = order_key(mine[(long long)g * n + i]);
+      gt += key > T;
+      eq += key == T;
+    }
+    gt = __reduce_add_sync(0xffffffffu, gt);
+    eq = __reduce_add_sync(0xffffffffu, eq);
+    if (lane == 0) {
+      if (gt) atomicAdd(&sh.cnt_gt[g], gt);
+      if (eq) atomicAdd(&sh.cnt_eq[g], eq);
+    }
+  }
+  cluster.sync();
+  if (rank == 0 && tid == 0) {
+    uint32_t rem = r;
+    for (int q = 0; q < cs; ++q) {
+      const uint32_t* pgt = cluster.map_shared_rank(sh.cnt_gt, q);
+      const uint32_t* peq = cluster.map_shared_rank(sh.cnt_eq, q);
+      for (int g = 0; g < heads; ++g) {
+        const uint32_t take = min(peq[g], rem);
+        out[q * heads + g] = (int32_t)min((long long)pgt[g] + take + floor_b, (long long)n);
+        rem -= take;
+      }
+    }
+  }
+  cluster.sync();   // rank 0 has read the peers' counts
+}
+
 }  // namespace
 
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
@@ -289,8 +405,30 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
   *launches += 1;
   const int32_t* budgets = nullptr;
   if (d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
-    adaptive_budget_kernel<<<d.nb, kSelThreads, 0, st>>>(ws.a, ws.budgets, d.Hkv, d.n, d.budget - d.Hkv * d.floor_b,
-                                                         (int)d.floor_b);
+    const long long b_adapt = d.budget - d.Hkv * d.floor_b;
+    int cs = 8;
+    while (cs > 1 && d.Hkv % cs != 0) cs >>= 1;
+    bool launched = false;
+    if (cs > 1) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)(d.nb * cs));
+      cfg.blockDim = dim3(kSelThreads);
+      cfg.dynamicSmemBytes = 0;
+      cfg.stream = st;
+      cudaLaunchAttribute attr;
+      attr.id = cudaLaunchAttributeClusterDimension;
+      attr.val.clusterDim.x = (unsigned)cs;
+      attr.val.clusterDim.y = 1;
+      attr.val.clusterDim.z = 1;
+      cfg.attrs = &attr;
+      cfg.numAttrs = 1;
+      const cudaError_t ec = cudaLaunchKernelEx(&cfg, adaptive_budget_cluster_kernel, (const float*)ws.a, ws.budgets,
+                                                d.Hkv, d.n, b_adapt, (int)d.floor_b);
+      if (ec == cudaSuccess) launched = true;
+      else (void)cudaGetLastError();   // no cluster launch on this device: use the single-CTA kernel
+    }
+    if (!launched)
+      adaptive_budget_kernel<<<d.nb, kSelThreads, 0, st>>>(ws.a, ws.budgets, d.Hkv, d.n, b_adapt, (int)d.floor_b);
     *launches += 1;
     budgets = ws.budgets;
   } else if (d.budget_mode == CKV_BUDGET_GIVEN) {

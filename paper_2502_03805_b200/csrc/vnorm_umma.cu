@@ -153,15 +153,9 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
           if (!mbar_wait_bounded(b_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
           mbar_arrive_expect_tx(b_full(s), L::kBStage);
           const uint32_t dst = sbase + L::kBOff + s * L::kBStage;
-#ifdef CKV_VN_B_KMAJOR
-#pragma unroll
-          for (int p = 0; p < kPanels; ++p)
-            tma_load_4d(dst + p * (kNC * 128), &mapW, p * 64, j * kNC, w.h, bw, b_full(s));
-#else
 #pragma unroll
           for (int nbk = 0; nbk < kNC / 64; ++nbk)
             tma_load_4d(dst + nbk * (DH * 128), &mapW, j * kNC + nbk * 64, 0, w.h, bw, b_full(s));
-#endif
           armed |= 1u << s;
           last_phase = (last_phase & ~(1u << s)) | (ph << s);
         }
@@ -203,11 +197,7 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-#ifdef CKV_VN_B_KMAJOR
-      constexpr uint32_t idesc = idesc_bf16_f32(128, kNC, 0);
-#else
       constexpr uint32_t idesc = idesc_bf16_f32(128, kNC, 1);
-#endif
       uint32_t it_b = 0, item_cnt = 0;
       uint32_t use[kTiles];
 #pragma unroll
@@ -234,11 +224,7 @@ vnorm_umma_kernel(const __grid_constant__ CUtensorMap mapV, const __grid_constan
                 //    next 64-element panel = next 128-row block.  B: N-major, 64-column blocks DH*128 bytes apart
                 //    (leading offset), 8-row K groups 1024 bytes apart (stride offset); 16 K rows = 2048 bytes.
                 const uint64_t ad = smem_desc_sw128(a_addr + (kk / 4) * (128 * 128) + (kk % 4) * 32, 16, 1024);
-#ifdef CKV_VN_B_KMAJOR
-                const uint64_t bd = smem_desc_sw128(b_addr + (kk / 4) * (kNC * 128) + (kk % 4) * 32, 16, 1024);
-#else
                 const uint64_t bd = smem_desc_sw128(b_addr + kk * 2048, DH * 128, 1024);
-#endif
                 umma_f16(tmem_base + m * kNC, ad, bd, idesc, kk > 0 ? 1u : 0u);
               }
               umma_commit(t_full(m));
@@ -351,16 +337,9 @@ cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, floa
   const cuuint32_t vbox[4] = {64, 128, 1, 1};
   if (!make_bf16_map_4d(&mv, V, vdims, vstr, vbox)) return cudaErrorNotSupported;
   const int nbw = d.wo_shared ? 1 : d.nb;
-#ifdef CKV_VN_B_KMAJOR
-  // experiment: WO given transposed, [nbw, Hq, dm, dh]
-  const cuuint64_t wdims[4] = {(cuuint64_t)d.dh, (cuuint64_t)d.dm, (cuuint64_t)d.Hq, (cuuint64_t)nbw};
-  const long long wstr[3] = {d.dh, (long long)d.dh * d.dm, (long long)d.Hq * d.dh * d.dm};
-  const cuuint32_t wbox[4] = {64, (cuuint32_t)kNC, 1, 1};
-#else
   const cuuint64_t wdims[4] = {(cuuint64_t)d.dm, (cuuint64_t)d.dh, (cuuint64_t)d.Hq, (cuuint64_t)nbw};
   const long long wstr[3] = {d.dm, (long long)d.dh * d.dm, (long long)d.Hq * d.dh * d.dm};
   const cuuint32_t wbox[4] = {64, (cuuint32_t)d.dh, 1, 1};
-#endif
   if (!make_bf16_map_4d(&mw, WO, wdims, wstr, wbox)) return cudaErrorNotSupported;
   UmmaArgs a;
   a.vnorm = vnorm; a.status = status_word;
