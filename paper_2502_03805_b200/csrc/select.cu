@@ -71,6 +71,21 @@ __device__ __forceinline__ bool excluded(const uint32_t* excl, long long i) {
   return excl != nullptr && ((excl[i >> 5] >> (i & 31)) & 1u);
 }
 
+// Applies f(index, value) to keys[0 .. count) with the CTA's threads striding over the array; eight independent loads
+// are issued before any of them is used, so the walk is not serialised on memory latency.
+template <typename F>
+__device__ __forceinline__ void scan_keys(const float* __restrict__ keys, long long count, F&& f) {
+  long long i = threadIdx.x;
+  for (; i + 7LL * kSelThreads < count; i += 8LL * kSelThreads) {
+    float v[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) v[q] = keys[i + (long long)q * kSelThreads];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) f(i + (long long)q * kSelThreads, v[q]);
+  }
+  for (; i < count; i += kSelThreads) f(i, keys[i]);
+}
+
 // Finds the k-th largest key among the candidates (all i in [0, count) not excluded), 1 <= k <= #candidates.
 // On return (all threads): *T = that key, *r = how many entries equal to T belong to the top k.
 __device__ void radix_select(const float* __restrict__ keys, long long count, const uint32_t* excl, uint32_t k,
@@ -83,11 +98,11 @@ __device__ void radix_select(const float* __restrict__ keys, long long count, co
     for (int e = tid; e < kSelWarps * 256; e += kSelThreads) (&sh.hist[0][0])[e] = 0;
     __syncthreads();
     const uint32_t prefix = sh.prefix;
-    for (long long i = tid; i < count; i += kSelThreads) {
-      if (excluded(excl, i)) continue;
-      const uint32_t key = order_key(keys[i]);
+    scan_keys(keys, count, [&](long long i, float x) {
+      if (excluded(excl, i)) return;
+      const uint32_t key = order_key(x);
       if ((key & known) == prefix) atomicAdd(&sh.hist[warp][(key >> shift) & 255u], 1u);
-    }
+    });
     __syncthreads();
     if (tid < 256) {
       uint32_t s = 0;
@@ -136,26 +151,45 @@ __device__ void mark_selected(const float* __restrict__ keys, int n, const uint3
   const int wpw = (nwords + kSelWarps - 1) / kSelWarps;
   const int w0 = min(warp * wpw, nwords), w1 = min(w0 + wpw, nwords);
   uint32_t eq_count = 0;
-  for (int q = w0; q < w1; ++q) {
-    const int i = q * 32 + lane;
-    const bool valid = any && i < n && !excluded(excl, i);
-    const bool eq = valid && order_key(keys[i]) == T;
-    eq_count += __popc(__ballot_sync(0xffffffffu, eq));
+  for (int q0 = w0; q0 < w1; q0 += 4) {
+    float x[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {   // independent loads first
+      const int i = (q0 + u) * 32 + lane;
+      x[u] = (any && q0 + u < w1 && i < n) ? keys[i] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = (q0 + u) * 32 + lane;
+      const bool valid = any && q0 + u < w1 && i < n && !excluded(excl, i);
+      eq_count += __popc(__ballot_sync(0xffffffffu, valid && order_key(x[u]) == T));
+    }
   }
   if (lane == 0) sh.warp_cnt[warp] = eq_count;
   __syncthreads();
   uint32_t running = 0;
   for (int q = 0; q < warp; ++q) running += sh.warp_cnt[q];
-  for (int q = w0; q < w1; ++q) {
-    const int i = q * 32 + lane;
-    const bool valid = any && i < n && !excluded(excl, i);
-    const uint32_t key = valid ? order_key(keys[i]) : 0u;
-    const bool eq = valid && key == T;
-    const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
-    const bool take = eq && (running + __popc(eqm & ((1u << lane) - 1u)) < r);
-    const uint32_t word = __ballot_sync(0xffffffffu, (valid && key > T) || take);
-    if (lane == 0) out[q] = word;
-    running += __popc(eqm);
+  for (int q0 = w0; q0 < w1; q0 += 4) {
+    float x[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = (q0 + u) * 32 + lane;
+      x[u] = (any && q0 + u < w1 && i < n) ? keys[i] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int q = q0 + u;
+      if (q >= w1) break;   // uniform across the warp
+      const int i = q * 32 + lane;
+      const bool valid = any && i < n && !excluded(excl, i);
+      const uint32_t key = valid ? order_key(x[u]) : 0u;
+      const bool eq = valid && key == T;
+      const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
+      const bool take = eq && (running + __popc(eqm & ((1u << lane) - 1u)) < r);
+      const uint32_t word = __ballot_sync(0xffffffffu, (valid && key > T) || take);
+      if (lane == 0) out[q] = word;
+      running += __popc(eqm);
+    }
   }
   __syncthreads();
 }
@@ -257,11 +291,11 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_kernel(const floa
   __syncthreads();
   for (int g = 0; g < Hkv; ++g) {
     uint32_t gt = 0, eq = 0;
-    for (int i = threadIdx.x; i < n; i += kSelThreads) {
-      const uint32_t key = order_key(ab[(long long)g * n + i]);
+    scan_keys(ab + (long long)g * n, n, [&](long long, float x) {
+      const uint32_t key = order_key(x);
       gt += key > T;
       eq += key == T;
-    }
+    });
     gt = __reduce_add_sync(0xffffffffu, gt);
     eq = __reduce_add_sync(0xffffffffu, eq);
     if ((threadIdx.x & 31) == 0) {
@@ -318,10 +352,10 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(co
     for (int e = tid; e < kSelWarps * 256; e += kSelThreads) (&sh.hist[0][0])[e] = 0;
     __syncthreads();
     const uint32_t prefix = sh.prefix;
-    for (long long i = tid; i < count; i += kSelThreads) {
-      const uint32_t key = order_key(mine[i]);
+    scan_keys(mine, count, [&](long long, float x) {
+      const uint32_t key = order_key(x);
       if ((key & known) == prefix) atomicAdd(&sh.hist[warp][(key >> shift) & 255u], 1u);
-    }
+    });
     __syncthreads();
     if (tid < 256) {
       uint32_t s = 0;
@@ -366,11 +400,11 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(co
   __syncthreads();
   for (int g = 0; g < heads; ++g) {
     uint32_t gt = 0, eq = 0;
-    for (int i = tid; i < n; i += kSelThreads) {
-      const uint32_t key = order_key(mine[(long long)g * n + i]);
+    scan_keys(mine + (long long)g * n, n, [&](long long, float x) {
+      const uint32_t key = order_key(x);
       gt += key > T;
       eq += key == T;
-    }
+    });
     gt = __reduce_add_sync(0xffffffffu, gt);
     eq = __reduce_add_sync(0xffffffffu, eq);
     if (lane == 0) {
