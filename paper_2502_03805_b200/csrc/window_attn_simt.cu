@@ -137,15 +137,27 @@ __global__ void attn_combine_kernel(const float* part_m, const float* part_l, fl
   rowstat[2 * r + 1] = 1.0f / (L * (float)w);
 }
 
-__global__ void maxpool_kernel(const float* __restrict__ abar, float* __restrict__ attn, int n, int kp) {
+// A CTA pools 1024 consecutive positions of one row from a shared-memory copy (with a halo of (kp-1)/2 on both sides),
+// so every input is read from global memory once.
+constexpr int kPoolTile = 1024;
+__global__ void __launch_bounds__(256) maxpool_kernel(const float* __restrict__ abar, float* __restrict__ attn, int n,
+                                                      int kp) {
+  __shared__ float tile[kPoolTile + 64];
   const long long base = (long long)blockIdx.y * n;
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  const int r = (kp - 1) / 2;
-  const int lo = max(i - r, 0), hi = min(i + r, n - 1);
-  float m = abar[base + lo];
-  for (int k = lo + 1; k <= hi; ++k) m = fmaxf(m, abar[base + k]);
-  attn[base + i] = m;
+  const int r = (kp - 1) / 2;          // <= 31
+  const int i0 = blockIdx.x * kPoolTile;
+  for (int e = threadIdx.x; e < kPoolTile + 2 * r; e += 256) {
+    const int i = i0 - r + e;
+    tile[e] = (i >= 0 && i < n) ? abar[base + i] : -INFINITY;   // outside the sequence: never the maximum
+  }
+  __syncthreads();
+  for (int e = threadIdx.x; e < kPoolTile; e += 256) {
+    const int i = i0 + e;
+    if (i >= n) break;
+    float m = tile[e];
+    for (int k = 1; k <= 2 * r; ++k) m = fmaxf(m, tile[e + k]);
+    attn[base + i] = m;
+  }
 }
 
 template <typename T, int DH, int WT>
@@ -161,7 +173,7 @@ cudaError_t run(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, 
   const int rows = d.nb * d.Hq * d.w;
   attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
   k2<<<grid, kThreads, smem, st>>>(a);
-  dim3 pgrid((d.n + 255) / 256, d.nb * d.Hq);
+  dim3 pgrid((d.n + kPoolTile - 1) / kPoolTile, d.nb * d.Hq);
   maxpool_kernel<<<pgrid, 256, 0, st>>>(a.abar, attn, d.n, d.kp);
   *launches += 4;
   return cudaGetLastError();
@@ -205,7 +217,7 @@ cudaError_t launch_attn_combine(const float* part_m, const float* part_l, float*
 }
 
 cudaError_t launch_maxpool(const float* abar, float* attn, int n, int kp, int nrows, cudaStream_t st) {
-  dim3 pgrid((n + 255) / 256, nrows);
+  dim3 pgrid((n + kPoolTile - 1) / kPoolTile, nrows);
   maxpool_kernel<<<pgrid, 256, 0, st>>>(abar, attn, n, kp);
   return cudaGetLastError();
 }
