@@ -141,6 +141,25 @@ CKV_API int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, con
                               size_t ws_bytes, void* stream);
 
 /*
+ * The two front steps of criticalkv_select on their own, for a layer whose KV heads are spread over several GPUs
+ * (each GPU holds some KV heads, their query heads and their rows of W^O).  Uniform budgets need nothing from other
+ * GPUs.  The flattened adaptive allocation (Algorithm 2, budget allocation) ranks the group attention scores of ALL
+ * heads of the layer, so each GPU
+ *   1. criticalkv_score on its heads, then criticalkv_group_scores: a_out[nb,Hkv_local,n] (and c_out, which may be
+ *      NULL) from attn and vnorm exactly as criticalkv_select computes them;
+ *   2. all-gathers a over the head axis (the caller's collective: Hkv*n floats per layer);
+ *   3. criticalkv_allocate_budgets with the descriptor of the WHOLE layer (Hkv, budget = B_total, CKV_BUDGET_FLAT_
+ *      ADAPTIVE; Hq, dh, dm only need to be consistent): budgets_out[nb,Hkv] int32, identical on every GPU;
+ *   4. criticalkv_select with its local descriptor in CKV_BUDGET_GIVEN mode and its slice of the budgets.
+ * The result equals, head for head, that of one GPU holding the whole layer.  All pointers are device memory,
+ * a/attn/vnorm 16-byte aligned; neither call needs a workspace.
+ */
+CKV_API int criticalkv_group_scores(criticalkv_handle h, const criticalkv_desc* d, const float* attn,
+                                    const float* vnorm, float* a_out, float* c_out, void* stream);
+CKV_API int criticalkv_allocate_budgets(criticalkv_handle h, const criticalkv_desc* d, const float* a,
+                                        int32_t* budgets_out, void* stream);
+
+/*
  * Allocation-free variant of criticalkv_select (the paper has no counterpart: this is a packaging of steps 3-4 for
  * callers that cannot provide a workspace).  Some hosts of this library may not allocate device memory at the point
  * where they compress a cache: a serving engine that reserved all of HBM for its own pools at start-up has nothing

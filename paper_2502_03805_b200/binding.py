@@ -22,7 +22,8 @@ CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM, CKV_FLAG_PROTECT
 CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",
-           "criticalkv_select", "criticalkv_select_static", "criticalkv_compact", "criticalkv_gather_positions", "criticalkv_compress",
+           "criticalkv_select", "criticalkv_group_scores", "criticalkv_allocate_budgets",
+           "criticalkv_select_static", "criticalkv_compact", "criticalkv_gather_positions", "criticalkv_compress",
            "criticalkv_host_staging_bytes", "criticalkv_compress_host", "criticalkv_selftest_bounded_wait",
            "criticalkv_diagnose_workspace_bytes", "criticalkv_diagnose", "criticalkv_device_status",
            "criticalkv_status_string", "criticalkv_last_cuda_error", "criticalkv_last_path",
@@ -65,6 +66,8 @@ def load():
     lib.criticalkv_workspace_bytes.argtypes = [dp, C.POINTER(sz), C.POINTER(sz)]
     lib.criticalkv_score.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.criticalkv_select.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.criticalkv_group_scores.argtypes = [vp, dp, vp, vp, vp, vp, vp]
+    lib.criticalkv_allocate_budgets.argtypes = [vp, dp, vp, vp, vp]
     lib.criticalkv_select_static.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
     lib.criticalkv_compact.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, vp]
     lib.criticalkv_gather_positions.argtypes = [vp, dp, vp, vp, vp, vp, vp]
@@ -170,6 +173,17 @@ def criticalkv_select(handle, desc, attn, vnorm, budgets_in, idx, offsets, stage
     rc = load().criticalkv_select(handle, C.byref(desc), _ptr(attn), _ptr(vnorm), _ptr(budgets_in), _ptr(idx),
                                   _ptr(offsets), _ptr(stage), _ptr(ws), _nbytes(ws, ws_bytes), _stream(stream))
     return _check(handle, rc, "criticalkv_select", check)
+
+
+def criticalkv_group_scores(handle, desc, attn, vnorm, a_out, c_out=None, stream=None, check=True):
+    rc = load().criticalkv_group_scores(handle, C.byref(desc), _ptr(attn), _ptr(vnorm), _ptr(a_out), _ptr(c_out),
+                                        _stream(stream))
+    return _check(handle, rc, "criticalkv_group_scores", check)
+
+
+def criticalkv_allocate_budgets(handle, desc, a, budgets_out, stream=None, check=True):
+    rc = load().criticalkv_allocate_budgets(handle, C.byref(desc), _ptr(a), _ptr(budgets_out), _stream(stream))
+    return _check(handle, rc, "criticalkv_allocate_budgets", check)
 
 
 def criticalkv_select_static(handle, desc, attn, vnorm, budgets_in, idx, offsets, stage, stream=None, check=True):

@@ -316,6 +316,39 @@ int criticalkv_compact(criticalkv_handle h, const criticalkv_desc* d, const void
   return record_cuda(h, e);
 }
 
+int criticalkv_group_scores(criticalkv_handle h, const criticalkv_desc* d, const float* attn, const float* vnorm,
+                            float* a_out, float* c_out, void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (!attn || !vnorm || !a_out) return CKV_EINVAL;
+  if (!aligned16(attn) || !aligned16(vnorm) || !aligned16(a_out) || !aligned16(c_out)) return CKV_EALIGN;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  int launches = 0;
+  cudaError_t e = ckv::launch_group_scores(dd, attn, vnorm, a_out, c_out, (cudaStream_t)stream, &launches);
+  h->launches += launches;
+  return record_cuda(h, e);
+}
+
+int criticalkv_allocate_budgets(criticalkv_handle h, const criticalkv_desc* d, const float* a, int32_t* budgets_out,
+                                void* stream) {
+  if (!h) return CKV_EINVAL;
+  Dims dd;
+  int rc = resolve(d, &dd);
+  if (rc != CKV_OK) return rc;
+  if (dd.budget_mode != CKV_BUDGET_FLAT_ADAPTIVE) return CKV_EINVAL;
+  if (!a || !budgets_out) return CKV_EINVAL;
+  if (!aligned16(a) || (reinterpret_cast<uintptr_t>(budgets_out) & 3u)) return CKV_EALIGN;
+  DeviceGuard guard(h->device);
+  if (!guard.ok) return CKV_ECUDA;
+  int launches = 0;
+  cudaError_t e = ckv::launch_allocate_budgets(dd, a, budgets_out, (cudaStream_t)stream, &launches);
+  h->launches += launches;
+  return record_cuda(h, e);
+}
+
 int criticalkv_gather_positions(criticalkv_handle h, const criticalkv_desc* d, const int32_t* pos_in,
                                 const int32_t* idx, const int32_t* offsets, int32_t* pos_out, void* stream) {
   if (!h) return CKV_EINVAL;

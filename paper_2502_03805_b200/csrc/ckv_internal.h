@@ -73,6 +73,12 @@ size_t vnorm_l2_workspace_bytes(const Dims& d);
 cudaError_t launch_vnorm_l2(const Dims& d, const void* V, const void* WO, float* vnorm, void* gram, int sm_count,
                             int cc_major, bool force_simt, int* status_word, cudaStream_t st, int* launches,
                             int* used_tensor_cores);
+// The two front steps of launch_select on their own (a layer whose KV heads live on several GPUs runs them around an
+// all-gather): group scores a (and c unless null), and the flattened adaptive allocation over a[nb, Hkv, n].
+cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* vnorm, float* a, float* c,
+                                cudaStream_t st, int* launches);
+cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* budgets_out, cudaStream_t st,
+                                    int* launches);
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word);

@@ -56,7 +56,7 @@ __global__ void group_reduce_kernel(const float* __restrict__ attn, const float*
   if (cv == 0.f) cv = 0.f;
   const long long o = ((long long)b * Hkv + g) * n + i;
   a[o] = av;
-  c[o] = cv;
+  if (c != nullptr) c[o] = cv;
 }
 
 struct SelectShared {
@@ -430,40 +430,53 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(co
 
 }  // namespace
 
+cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* vnorm, float* a, float* c,
+                                cudaStream_t st, int* launches) {
+  dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
+  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, a, c, d.Hq, d.Hkv, d.G, d.n, d.eps, d.group_sum,
+                                             d.protect_window ? d.n - d.w : d.n);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
+cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* budgets_out, cudaStream_t st,
+                                    int* launches) {
+  const long long b_adapt = d.budget - d.Hkv * d.floor_b;
+  int cs = 8;
+  while (cs > 1 && d.Hkv % cs != 0) cs >>= 1;
+  bool launched = false;
+  if (cs > 1) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(d.nb * cs));
+    cfg.blockDim = dim3(kSelThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = (unsigned)cs;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    const cudaError_t ec = cudaLaunchKernelEx(&cfg, adaptive_budget_cluster_kernel, a_all, budgets_out, d.Hkv, d.n,
+                                              b_adapt, (int)d.floor_b);
+    if (ec == cudaSuccess) launched = true;
+    else (void)cudaGetLastError();   // no cluster launch on this device: use the single-CTA kernel
+  }
+  if (!launched)
+    adaptive_budget_kernel<<<d.nb, kSelThreads, 0, st>>>(a_all, budgets_out, d.Hkv, d.n, b_adapt, (int)d.floor_b);
+  *launches += 1;
+  return cudaGetLastError();
+}
+
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           cudaStream_t st, int* launches, int* status_word) {
-  dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
-  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, ws.a, ws.c, d.Hq, d.Hkv, d.G, d.n, d.eps, d.group_sum,
-                                             d.protect_window ? d.n - d.w : d.n);
-  *launches += 1;
+  cudaError_t e = launch_group_scores(d, attn, vnorm, ws.a, ws.c, st, launches);
+  if (e != cudaSuccess) return e;
   const int32_t* budgets = nullptr;
   if (d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
-    const long long b_adapt = d.budget - d.Hkv * d.floor_b;
-    int cs = 8;
-    while (cs > 1 && d.Hkv % cs != 0) cs >>= 1;
-    bool launched = false;
-    if (cs > 1) {
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((unsigned)(d.nb * cs));
-      cfg.blockDim = dim3(kSelThreads);
-      cfg.dynamicSmemBytes = 0;
-      cfg.stream = st;
-      cudaLaunchAttribute attr;
-      attr.id = cudaLaunchAttributeClusterDimension;
-      attr.val.clusterDim.x = (unsigned)cs;
-      attr.val.clusterDim.y = 1;
-      attr.val.clusterDim.z = 1;
-      cfg.attrs = &attr;
-      cfg.numAttrs = 1;
-      const cudaError_t ec = cudaLaunchKernelEx(&cfg, adaptive_budget_cluster_kernel, (const float*)ws.a, ws.budgets,
-                                                d.Hkv, d.n, b_adapt, (int)d.floor_b);
-      if (ec == cudaSuccess) launched = true;
-      else (void)cudaGetLastError();   // no cluster launch on this device: use the single-CTA kernel
-    }
-    if (!launched)
-      adaptive_budget_kernel<<<d.nb, kSelThreads, 0, st>>>(ws.a, ws.budgets, d.Hkv, d.n, b_adapt, (int)d.floor_b);
-    *launches += 1;
+    if ((e = launch_allocate_budgets(d, ws.a, ws.budgets, st, launches)) != cudaSuccess) return e;
     budgets = ws.budgets;
   } else if (d.budget_mode == CKV_BUDGET_GIVEN) {
     budgets = budgets_in;
@@ -473,7 +486,7 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
   p.status = status_word;
   p.Hkv = d.Hkv; p.n = d.n; p.uniform_b = d.budget; p.btot = d.btot; p.alpha = d.alpha;
   const size_t dyn = (size_t)2 * ((d.n + 31) / 32) * sizeof(uint32_t);
-  cudaError_t e = cudaFuncSetAttribute(two_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
+  e = cudaFuncSetAttribute(two_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
   if (e != cudaSuccess) return e;
   dim3 tgrid(d.Hkv, d.nb);
   two_stage_kernel<<<tgrid, kSelThreads, dyn, st>>>(p);

@@ -42,5 +42,41 @@ def test_two_ranks_take_the_max_time_and_own_disjoint_layers():
     assert whole_job_throughput(1000, 2, 0.015) == 2000 / 0.015
 
 
+def _gather_worker(rank, world, port, out):
+    import torch
+    from paper_2502_03805_b200.dist_util import all_gather_heads, shard_kv_heads
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    g0, g1 = shard_kv_heads(8, world, rank)
+    full = torch.arange(2 * 8 * 5, dtype=torch.float32).reshape(2, 8, 5)
+    got = all_gather_heads(full[:, g0:g1].contiguous())
+    out.put((rank, (g0, g1), bool(torch.equal(got, full))))
+    dist.destroy_process_group()
+
+
+def test_kv_head_shards_gather_back_in_head_order():
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_gather_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert res == [(0, (0, 4), True), (1, (4, 8), True)]
+
+
+def test_kv_head_shards_reject_uneven_splits():
+    import pytest
+    from paper_2502_03805_b200.dist_util import shard_kv_heads
+    assert [shard_kv_heads(8, 4, r) for r in range(4)] == [(0, 2), (2, 4), (4, 6), (6, 8)]
+    with pytest.raises(ValueError):
+        shard_kv_heads(8, 3, 0)
+    with pytest.raises(ValueError):
+        shard_kv_heads(8, 2, 2)
+
+
 def test_single_process_is_identity():
     assert max_over_ranks(3.5) == 3.5

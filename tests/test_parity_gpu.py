@@ -322,6 +322,42 @@ def test_l2_norm_variant(kw, tensor_cores):
         pu.check_layer_against_oracle(L, wl, out, norm="l2")
 
 
+@pytest.mark.parametrize("world", [2, 4])
+def test_kv_head_sharded_adaptive_compression_equals_unsharded(world):
+    # the ranks of a KV-head-sharded layer are played one after the other on this GPU; the all-gather of the group
+    # scores is a concatenation.  Every rank must end up with exactly the rows the unsharded call keeps for its heads.
+    from paper_2502_03805_b200 import to_device, to_host
+    from paper_2502_03805_b200.dist_util import ShardedCompressor
+    wl = small_workload(cfg_id=210, dtype="bf16", n=1800, w=32, kp=7, budget_mode="adaptive", budget=1500, dh=128,
+                        dm=512, Hq=16, Hkv=4)
+    Ls, full, _ = _run(wl)
+    L, ref = Ls[0], full[0]
+    shards, a_parts = [], []
+    for rank in range(world):
+        sc = ShardedCompressor(nb=1, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp,
+                               dtype="bf16", budget_mode="adaptive", budget=wl.budget, world=world, rank=rank)
+        g0, g1 = sc.g0, sc.g1
+        h0, h1 = g0 * wl.G, g1 * wl.G
+        t = [to_device(np.ascontiguousarray(x)[None], "bf16")
+             for x in (L.Qw_store[h0:h1], L.K_store[g0:g1], L.V_store[g0:g1], L.WO_store[h0:h1])]
+        sc.session.score(*t)
+        a_parts.append(sc.group_scores().clone())
+        shards.append((sc, t))
+    a_all = torch.cat(a_parts, dim=1)
+    for sc, t in shards:
+        sc.gather = lambda a, a_all=a_all: a_all
+        s = sc.compress(*t)
+        torch.cuda.synchronize()
+        assert s.device_status() == 0
+        g0, g1 = sc.g0, sc.g1
+        off = to_host(s.offsets[0])
+        np.testing.assert_array_equal(np.diff(off), np.diff(ref["offsets"])[g0:g1])
+        lo, hi = ref["offsets"][g0], ref["offsets"][g1]
+        np.testing.assert_array_equal(to_host(s.idx[0])[: off[-1]], ref["idx"][lo:hi])
+        np.testing.assert_array_equal(to_host(s.K_out[0])[: off[-1]], ref["K_out"][lo:hi])
+        np.testing.assert_array_equal(to_host(s.V_out[0])[: off[-1]], ref["V_out"][lo:hi])
+
+
 def test_bounded_wait_times_out_and_reports_status():
     # a wait on a barrier nothing signals must end by itself, set CKV_ETIMEOUT, and leave the context usable
     import time
