@@ -87,7 +87,7 @@ typedef struct {
   int32_t dh;            /* head dim: 64 or 128                                                         */
   int32_t dm;            /* model dim, multiple of 8                                                    */
   int32_t n;             /* cached entries per head, >= w                                               */
-  int32_t w;             /* observation window (Algorithm 2: n'), 1..64                                 */
+  int32_t w;             /* observation window (Algorithm 2: n'), 1..256 (criticalkv_diagnose: 1..64)   */
   int32_t pool_k;        /* max-pool kernel, odd, 1..63 (Algorithm 2: maxpooling; 7 in the paper)       */
   int32_t dtype;         /* criticalkv_dtype of Qw, K, V, WO, K_out, V_out                              */
   float scale;           /* logit scale of Eq. 2; <= 0 selects 1/sqrt(dh)                               */
@@ -222,8 +222,8 @@ CKV_API int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc*
  *   diag[nb,Hq,w,10] = sigma (attention mass of the stage-1 set, Assumption 3.4), retained mass, C = sum_i A_i nu_i,
  *   its parts over stage 1 and stage 2, min_i nu_i, L = ||(A - A') V W^O||_1 (Definition 3.1 with A' of Theorem 3.2),
  *   theta (Theorem 3.3), theta_hat (Theorem 3.5), theta_relax (relaxed bound of the appendix).
- * vnorm is the per-head output of criticalkv_score (not available with CKV_FLAG_WO_GROUP_SUM); idx, offsets and
- * stage (required) come from criticalkv_select.  ws: criticalkv_diagnose_workspace_bytes, 256-byte aligned.
+ * vnorm is the per-head output of criticalkv_score (CKV_ENOTSUP with CKV_FLAG_WO_GROUP_SUM or w > 64); idx, offsets
+ * and stage (required) come from criticalkv_select.  ws: criticalkv_diagnose_workspace_bytes, 256-byte aligned.
  */
 #define CKV_DIAG_FIELDS 10
 CKV_API int criticalkv_diagnose_workspace_bytes(const criticalkv_desc* d, size_t* bytes);

@@ -44,7 +44,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (d->dh != 64 && d->dh != 128) return CKV_ENOTSUP;
   if (d->dm < 8 || d->dm % 8 != 0) return CKV_EINVAL;
   if (d->w < 1) return CKV_EINVAL;
-  if (d->w > 64) return CKV_ENOTSUP;
+  if (d->w > 256) return CKV_ENOTSUP;
   if (d->n < d->w) return CKV_EINVAL;
   if (d->pool_k < 1 || d->pool_k % 2 == 0) return CKV_EINVAL;
   if (d->pool_k > 63) return CKV_ENOTSUP;
@@ -538,6 +538,7 @@ int criticalkv_diagnose(criticalkv_handle h, const criticalkv_desc* d, const voi
   int rc = resolve(d, &dd);
   if (rc != CKV_OK) return rc;
   if (dd.group_sum) return CKV_ENOTSUP;  // the bounds are stated with per-head norms
+  if (dd.w > 64) return CKV_ENOTSUP;     // the diagnostics kernel keeps a window's rows in registers
   if (!Qw || !K || !V || !WO || !vnorm || !idx || !offsets || !stage || !diag || !ws) return CKV_EINVAL;
   if (!aligned16(Qw) || !aligned16(K) || !aligned16(V) || !aligned16(WO) || !aligned16(vnorm) || !aligned16(diag) ||
       (reinterpret_cast<uintptr_t>(idx) & 3u) || (reinterpret_cast<uintptr_t>(offsets) & 3u) ||

@@ -31,11 +31,12 @@ struct AttnArgs {
   long long qs[3], ks[3];
 };
 
+// Window rows j0 .. j0+WT-1 of query head h as floats; rows past w are zero-filled.
 template <typename T, int DH, int WT>
-__device__ __forceinline__ void stage_queries(const AttnArgs& a, int b, int h, float* q_s) {
+__device__ __forceinline__ void stage_queries(const AttnArgs& a, int b, int h, int j0, float* q_s) {
   const T* q = reinterpret_cast<const T*>(a.Qw) + b * a.qs[0] + h * a.qs[1];
   for (int e = threadIdx.x; e < WT * DH; e += kThreads) {
-    int j = e / DH, t = e % DH;
+    int j = j0 + e / DH, t = e % DH;
     q_s[e] = (j < a.w) ? to_float(q[j * a.qs[2] + t]) : 0.f;
   }
 }
@@ -51,72 +52,79 @@ __global__ void __launch_bounds__(kThreads) attn_pass_kernel(AttnArgs a) {
   const int i = chunk * kAttnChunk + threadIdx.x;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-  stage_queries<T, DH, WT>(a, b, h, q_s);
   const long long row = (long long)(b * a.Hq + h) * a.w;
-  if constexpr (kProb) {
-    for (int e = threadIdx.x; e < 2 * a.w; e += kThreads) stat[e] = a.rowstat[row * 2 + e];
-  }
-  __syncthreads();
-
-  float acc[WT];
   const bool in_range = i < a.n;
-  if (in_range) {
-    const T* krow = reinterpret_cast<const T*>(a.K) + b * a.ks[0] + g * a.ks[1] + (long long)i * a.ks[2];
-    key_logits<T, DH, WT>(krow, q_s, acc);
-  } else {
-#pragma unroll
-    for (int j = 0; j < WT; ++j) acc[j] = 0.f;
-  }
   const int first_pos = a.n - a.w;  // sequence position of window row 0
-#pragma unroll
-  for (int j = 0; j < WT; ++j) {
-    const bool visible = in_range && j < a.w && i <= first_pos + j;
-    acc[j] = visible ? acc[j] * a.scale : -INFINITY;
-  }
+  float s = 0.f;                    // second pass: sum of the normalised weights over the window rows
+  // the window is walked in blocks of WT rows (one block unless w > 64)
+  for (int j0 = 0; j0 < a.w; j0 += WT) {
+    if (j0 > 0) __syncthreads();    // the previous block's queries and scratch are no longer read
+    stage_queries<T, DH, WT>(a, b, h, j0, q_s);
+    const int wb = min(WT, a.w - j0);
+    if constexpr (kProb) {
+      for (int e = threadIdx.x; e < 2 * wb; e += kThreads) stat[e] = a.rowstat[(row + j0) * 2 + e];
+    }
+    __syncthreads();
 
-  if constexpr (kProb) {
-    // normalise with the final row statistics and sum the window rows in increasing row order
-    float s = 0.f;
+    float acc[WT];
+    if (in_range) {
+      const T* krow = reinterpret_cast<const T*>(a.K) + b * a.ks[0] + g * a.ks[1] + (long long)i * a.ks[2];
+      key_logits<T, DH, WT>(krow, q_s, acc);
+    } else {
+#pragma unroll
+      for (int j = 0; j < WT; ++j) acc[j] = 0.f;
+    }
 #pragma unroll
     for (int j = 0; j < WT; ++j) {
-      if (j < a.w) {
-        float p = (acc[j] == -INFINITY) ? 0.f : expf(acc[j] - stat[2 * j]) * stat[2 * j + 1];
-        s += p;
+      const bool visible = in_range && j < wb && i <= first_pos + j0 + j;
+      acc[j] = visible ? acc[j] * a.scale : -INFINITY;
+    }
+
+    if constexpr (kProb) {
+      // normalise with the final row statistics and sum the window rows in increasing row order
+#pragma unroll
+      for (int j = 0; j < WT; ++j) {
+        if (j < wb) {
+          float p = (acc[j] == -INFINITY) ? 0.f : expf(acc[j] - stat[2 * j]) * stat[2 * j + 1];
+          s += p;
+        }
+      }
+    } else {
+      // chunk maximum per row
+#pragma unroll
+      for (int j = 0; j < WT; ++j) {
+        float m = acc[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) red[warp * WT + j] = m;
+      }
+      __syncthreads();
+      if (threadIdx.x < WT) {
+        float m = red[threadIdx.x];
+        for (int wq = 1; wq < kThreads / 32; ++wq) m = fmaxf(m, red[wq * WT + threadIdx.x]);
+        stat[threadIdx.x] = m;
+      }
+      __syncthreads();
+      // chunk sum of exp(logit - chunk max)
+#pragma unroll
+      for (int j = 0; j < WT; ++j) {
+        float e = (acc[j] == -INFINITY) ? 0.f : expf(acc[j] - stat[j]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
+        if (lane == 0) red[warp * WT + j] = e;
+      }
+      __syncthreads();
+      if (threadIdx.x < wb) {
+        float l = red[threadIdx.x];
+        for (int wq = 1; wq < kThreads / 32; ++wq) l += red[wq * WT + threadIdx.x];
+        const long long o = (row + j0 + threadIdx.x) * a.nchunks + chunk;
+        a.part_m[o] = stat[threadIdx.x];
+        a.part_l[o] = l;
       }
     }
+  }
+  if constexpr (kProb) {
     if (in_range) a.abar[(long long)(b * a.Hq + h) * a.n + i] = s;
-  } else {
-    // chunk maximum per row
-#pragma unroll
-    for (int j = 0; j < WT; ++j) {
-      float m = acc[j];
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-      if (lane == 0) red[warp * WT + j] = m;
-    }
-    __syncthreads();
-    if (threadIdx.x < WT) {
-      float m = red[threadIdx.x];
-      for (int wq = 1; wq < kThreads / 32; ++wq) m = fmaxf(m, red[wq * WT + threadIdx.x]);
-      stat[threadIdx.x] = m;
-    }
-    __syncthreads();
-    // chunk sum of exp(logit - chunk max)
-#pragma unroll
-    for (int j = 0; j < WT; ++j) {
-      float e = (acc[j] == -INFINITY) ? 0.f : expf(acc[j] - stat[j]);
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) e += __shfl_xor_sync(0xffffffffu, e, o);
-      if (lane == 0) red[warp * WT + j] = e;
-    }
-    __syncthreads();
-    if (threadIdx.x < a.w) {
-      float l = red[threadIdx.x];
-      for (int wq = 1; wq < kThreads / 32; ++wq) l += red[wq * WT + threadIdx.x];
-      const long long o = (row + threadIdx.x) * a.nchunks + chunk;
-      a.part_m[o] = stat[threadIdx.x];
-      a.part_l[o] = l;
-    }
   }
 }
 

@@ -35,7 +35,7 @@ constexpr int kKeyTile = 128;
 constexpr int kHalves = 1;
 constexpr int kThreads = (2 + 8 * kHalves) * 32;
 constexpr int kSlotCols = 256;
-constexpr int kMaxRowBlocks = 3;  // G*w <= 384
+constexpr int kMaxRowBlocks = 3;  // query rows per work item <= 384
 constexpr float kLog2e = 1.4426950408889634f;
 
 enum { kStats = 1, kProbs = 2 };
@@ -47,13 +47,15 @@ struct AttnUmmaArgs {
   float* abar;
   int* status;
   int Hq, Hkv, G, n, nb;
-  int rows;            // G * w
+  int Gi;              // query heads per work item: the largest divisor of G with Gi * w <= 384
+  int subgroups;       // G / Gi work items share a KV head's key tiles
+  int rows;            // Gi * w
   int row_blocks;      // ceil(rows / 128)                          (sweep 1 sub-tiles per key tile)
   int heads_per_group; // heads per MMA in sweep 2 (hg * w <= 256)
-  int head_groups;     // ceil(G / heads_per_group)                 (sweep 2 sub-tiles per key tile)
+  int head_groups;     // ceil(Gi / heads_per_group)                (sweep 2 sub-tiles per key tile)
   int ntiles;          // ceil(n / 128)
   int tiles_per_item;
-  int chunks_per_bg;   // work items per (nb, KV head)
+  int chunks_per_bg;   // work items per (nb, KV head, subgroup)
   int part_stride;     // partial slots per row = 2 * chunks_per_bg
   int kstages;
   int qbufs;           // 1 or 2 shared-memory copies of the group's Q rows (and statistics)
@@ -64,13 +66,17 @@ struct AttnUmmaArgs {
 
 struct Item {
   int b, g, chunk, t0, t1;
+  int h0;   // first query head of the item
 };
 __device__ __forceinline__ Item decode_item(long long item, const AttnUmmaArgs& a) {
   Item it;
   it.chunk = (int)(item % a.chunks_per_bg);
-  const long long r = item / a.chunks_per_bg;
+  long long r = item / a.chunks_per_bg;
+  const int sg = (int)(r % a.subgroups);
+  r /= a.subgroups;
   it.g = (int)(r % a.Hkv);
   it.b = (int)(r / a.Hkv);
+  it.h0 = it.g * a.G + sg * a.Gi;
   it.t0 = it.chunk * a.tiles_per_item;
   it.t1 = min(it.t0 + a.tiles_per_item, a.ntiles);
   return it;
@@ -176,7 +182,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         // the normalisation constants of the group's rows, next to the Q buffer they belong to
         float* dst = stats + qb * a.rows;
         for (int r = lane; r < a.rows; r += 32) {
-          const long long rowg = ((long long)w.b * a.Hq + (long long)w.g * a.G + r / W) * W + r % W;
+          const long long rowg = ((long long)w.b * a.Hq + w.h0 + r / W) * W + r % W;
           dst[r] = fmaf(-a.rowstat[2 * rowg], kLog2e, log2f(a.rowstat[2 * rowg + 1]));
         }
         __syncwarp();
@@ -185,7 +191,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         mbar_arrive_expect_tx(q_full(qb), (uint32_t)(a.rows * DH * 2));
 #pragma unroll
         for (int p = 0; p < kPanels; ++p)
-          tma_load_4d(sbase + qb * L.q_bytes + p * L.q_panel, &mapQ, p * 64, 0, w.g * a.G, w.b, q_full(qb));
+          tma_load_4d(sbase + qb * L.q_bytes + p * L.q_panel, &mapQ, p * 64, 0, w.h0, w.b, q_full(qb));
         q_armed = true;
         q_last = (uint32_t)qb | (qph << 1);
         for (int t = w.t0; t < w.t1; ++t, ++it_k) {
@@ -237,7 +243,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
             } else {
               // rows = the 128 keys of the tile, columns = the window rows of this head group
               const int h0 = sub * a.heads_per_group;
-              const int ncols = min(a.heads_per_group, a.G - h0) * W;
+              const int ncols = min(a.heads_per_group, a.Gi - h0) * W;
               idesc = idesc_bf16_f32(128, ncols, 0);
               a_addr = k_addr;
               a_panel = kKeyTile * 128;
@@ -357,7 +363,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
           } else {
             const int i = key0 + quad * 32 + lane;               // this thread's key
             const int h0 = sub * a.heads_per_group;
-            const int nh = min(a.heads_per_group, a.G - h0);
+            const int nh = min(a.heads_per_group, a.Gi - h0);
             const int hph = (a.heads_per_group + kHalves - 1) / kHalves;   // heads per column half
             const int hq0 = half * hph, hq1 = min(nh, hq0 + hph);
             if (hq0 >= hq1) {
@@ -365,41 +371,45 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
               __syncwarp();
               if (lane == 0) mbar_arrive(t_empty(set));
             }
+            // the W weights of a (key, head) pair are read from tensor memory in chunks of at most 64 columns
+            constexpr int JC = W < 64 ? W : 64;
             for (int hq = hq0; hq < hq1; ++hq) {
-              float v[W / 16][16];
-#pragma unroll
-              for (int q = 0; q < W / 16; ++q) tmem_ld_16cols(lane_base + hq * W + q * 16, v[q]);
-              tc_wait_ld();
-              if (hq == hq1 - 1) {
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(t_empty(set));
-              }
-              // bias_j = -max_j * log2e + log2(1 / (w * sum_j)): one fma and one exp per weight
-              const float4* sr = reinterpret_cast<const float4*>(st + (h0 + hq) * W);
               float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-              if (!tail) {
+#pragma unroll 1
+              for (int jc = 0; jc < W; jc += JC) {
+                float v[JC / 16][16];
 #pragma unroll
-                for (int j = 0; j < W; j += 4) {
-                  const float4 bz = sr[j / 4];
-                  a0 += ex2_approx(fmaf(v[j / 16][j % 16], a.c, bz.x));
-                  a1 += ex2_approx(fmaf(v[(j + 1) / 16][(j + 1) % 16], a.c, bz.y));
-                  a2 += ex2_approx(fmaf(v[(j + 2) / 16][(j + 2) % 16], a.c, bz.z));
-                  a3 += ex2_approx(fmaf(v[(j + 3) / 16][(j + 3) % 16], a.c, bz.w));
+                for (int q = 0; q < JC / 16; ++q) tmem_ld_16cols(lane_base + hq * W + jc + q * 16, v[q]);
+                tc_wait_ld();
+                if (hq == hq1 - 1 && jc + JC >= W) {
+                  tc_fence_before();
+                  __syncwarp();
+                  if (lane == 0) mbar_arrive(t_empty(set));
                 }
-              } else {
-                const int jmin = i - first_pos;                   // rows j < jmin do not see key i
+                // bias_j = -max_j * log2e + log2(1 / (w * sum_j)): one fma and one exp per weight
+                const float4* sr = reinterpret_cast<const float4*>(st + (h0 + hq) * W + jc);
+                if (!tail) {
 #pragma unroll
-                for (int j = 0; j < W; j += 4) {
-                  const float4 bz = sr[j / 4];
-                  a0 += j >= jmin ? ex2_approx(fmaf(v[j / 16][j % 16], a.c, bz.x)) : 0.f;
-                  a1 += j + 1 >= jmin ? ex2_approx(fmaf(v[(j + 1) / 16][(j + 1) % 16], a.c, bz.y)) : 0.f;
-                  a2 += j + 2 >= jmin ? ex2_approx(fmaf(v[(j + 2) / 16][(j + 2) % 16], a.c, bz.z)) : 0.f;
-                  a3 += j + 3 >= jmin ? ex2_approx(fmaf(v[(j + 3) / 16][(j + 3) % 16], a.c, bz.w)) : 0.f;
+                  for (int j = 0; j < JC; j += 4) {
+                    const float4 bz = sr[j / 4];
+                    a0 += ex2_approx(fmaf(v[j / 16][j % 16], a.c, bz.x));
+                    a1 += ex2_approx(fmaf(v[(j + 1) / 16][(j + 1) % 16], a.c, bz.y));
+                    a2 += ex2_approx(fmaf(v[(j + 2) / 16][(j + 2) % 16], a.c, bz.z));
+                    a3 += ex2_approx(fmaf(v[(j + 3) / 16][(j + 3) % 16], a.c, bz.w));
+                  }
+                } else {
+                  const int jmin = i - first_pos - jc;              // rows jc + j with j < jmin do not see key i
+#pragma unroll
+                  for (int j = 0; j < JC; j += 4) {
+                    const float4 bz = sr[j / 4];
+                    a0 += j >= jmin ? ex2_approx(fmaf(v[j / 16][j % 16], a.c, bz.x)) : 0.f;
+                    a1 += j + 1 >= jmin ? ex2_approx(fmaf(v[(j + 1) / 16][(j + 1) % 16], a.c, bz.y)) : 0.f;
+                    a2 += j + 2 >= jmin ? ex2_approx(fmaf(v[(j + 2) / 16][(j + 2) % 16], a.c, bz.z)) : 0.f;
+                    a3 += j + 3 >= jmin ? ex2_approx(fmaf(v[(j + 3) / 16][(j + 3) % 16], a.c, bz.w)) : 0.f;
+                  }
                 }
               }
-              if (i < a.n)
-                a.abar[((long long)w.b * a.Hq + (long long)w.g * a.G + h0 + hq) * a.n + i] = (a0 + a1) + (a2 + a3);
+              if (i < a.n) a.abar[((long long)w.b * a.Hq + w.h0 + h0 + hq) * a.n + i] = (a0 + a1) + (a2 + a3);
             }
           }
         }
@@ -413,7 +423,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         for (int rb = 0; rb < kMaxRowBlocks; ++rb) {
           const int r = rb * 128 + quad * 32 + lane;
           if (rb < a.row_blocks && r < a.rows) {
-            const long long rowg = ((long long)w.b * a.Hq + (long long)w.g * a.G + r / W) * W + r % W;
+            const long long rowg = ((long long)w.b * a.Hq + w.h0 + r / W) * W + r % W;
             const long long o = rowg * a.part_stride + (w.chunk * 2 + set) * kHalves + half;
             a.part_m[o] = rm[rb] * a.scale;
             a.part_l[o] = rl[rb];
@@ -468,21 +478,27 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
                                     const ScoreWorkspace& ws, int sm_count, int* status_word, cudaStream_t st,
                                     int* launches) {
   if (d.dtype != CKV_BF16 || tma_encode_fn() == nullptr) return cudaErrorNotSupported;
-  if (d.w != 16 && d.w != 32 && d.w != 64) return cudaErrorNotSupported;
-  const int rows = d.G * d.w;
+  if (d.w != 16 && d.w != 32 && d.w != 64 && d.w != 128 && d.w != 256) return cudaErrorNotSupported;
+  // a work item covers Gi query heads of a KV head; with long windows the group is split and every part streams
+  // the KV head's keys again (from L2 when they are still there)
+  int Gi = d.G;
+  while (Gi > 1 && (d.G % Gi != 0 || Gi * d.w > 128 * kMaxRowBlocks)) --Gi;
+  const int rows = Gi * d.w;
   if (rows > 128 * kMaxRowBlocks) return cudaErrorNotSupported;
 
   AttnUmmaArgs a;
   a.part_m = ws.part_m; a.part_l = ws.part_l; a.rowstat = ws.rowstat; a.abar = ws.abar; a.status = status_word;
   a.Hq = d.Hq; a.Hkv = d.Hkv; a.G = d.G; a.n = d.n; a.nb = d.nb;
+  a.Gi = Gi;
+  a.subgroups = d.G / Gi;
   a.rows = rows;
   a.row_blocks = (rows + 127) / 128;
-  a.heads_per_group = kSlotCols / d.w < d.G ? kSlotCols / d.w : d.G;
-  a.head_groups = (d.G + a.heads_per_group - 1) / a.heads_per_group;
+  a.heads_per_group = kSlotCols / d.w < Gi ? kSlotCols / d.w : Gi;
+  a.head_groups = (Gi + a.heads_per_group - 1) / a.heads_per_group;
   a.ntiles = (d.n + kKeyTile - 1) / kKeyTile;
   // enough work items to fill the machine a few times over, but at least 4 key tiles each so that the partial
   // statistics (two per item) fit the workspace sized for one partial per 256 keys
-  const long long groups = (long long)d.nb * d.Hkv;
+  const long long groups = (long long)d.nb * d.Hkv * a.subgroups;
   long long want_items = 4LL * sm_count;
   int tpi = (int)((groups * a.ntiles + want_items - 1) / want_items);
   if (tpi < 4 * kHalves) tpi = 4 * kHalves;
@@ -507,7 +523,7 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
   CUtensorMap mq, mk;
   const cuuint64_t qdims[4] = {(cuuint64_t)d.dh, (cuuint64_t)d.w, (cuuint64_t)d.Hq, (cuuint64_t)d.nb};
   const long long qstr[3] = {d.qs[2], d.qs[1], d.qs[0]};
-  const cuuint32_t qbox[4] = {64, (cuuint32_t)d.w, (cuuint32_t)d.G, 1};
+  const cuuint32_t qbox[4] = {64, (cuuint32_t)d.w, (cuuint32_t)Gi, 1};
   if (!make_bf16_map_4d(&mq, Qw, qdims, qstr, qbox)) return cudaErrorNotSupported;
   const cuuint64_t kdims[4] = {(cuuint64_t)d.dh, (cuuint64_t)d.n, (cuuint64_t)d.Hkv, (cuuint64_t)d.nb};
   const long long kstr[3] = {d.ks[2], d.ks[1], d.ks[0]};
@@ -517,8 +533,8 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
   const int grid = (int)(a.nitems < sm_count ? a.nitems : sm_count);
 #define CKV_ATTN_CASE(DHV, WV) \
   if (d.dh == DHV && d.w == WV) return run_both<DHV, WV>(d, mq, mk, a, grid, attn, ws, st, launches);
-  CKV_ATTN_CASE(128, 16) CKV_ATTN_CASE(128, 32) CKV_ATTN_CASE(128, 64)
-  CKV_ATTN_CASE(64, 16) CKV_ATTN_CASE(64, 32) CKV_ATTN_CASE(64, 64)
+  CKV_ATTN_CASE(128, 16) CKV_ATTN_CASE(128, 32) CKV_ATTN_CASE(128, 64) CKV_ATTN_CASE(128, 128) CKV_ATTN_CASE(128, 256)
+  CKV_ATTN_CASE(64, 16) CKV_ATTN_CASE(64, 32) CKV_ATTN_CASE(64, 64) CKV_ATTN_CASE(64, 128) CKV_ATTN_CASE(64, 256)
 #undef CKV_ATTN_CASE
   return cudaErrorNotSupported;
 }

@@ -48,7 +48,7 @@ def test_workspace_bytes_are_sane(lib):
 
 @pytest.mark.parametrize("kw,status", [
     (dict(nb=0), B.CKV_EINVAL), (dict(Hq=5), B.CKV_EINVAL), (dict(dh=96), B.CKV_ENOTSUP),
-    (dict(dm=250), B.CKV_EINVAL), (dict(n=8), B.CKV_EINVAL), (dict(w=0), B.CKV_EINVAL), (dict(w=65, n=512), B.CKV_ENOTSUP),
+    (dict(dm=250), B.CKV_EINVAL), (dict(n=8), B.CKV_EINVAL), (dict(w=0), B.CKV_EINVAL), (dict(w=257, n=512), B.CKV_ENOTSUP),
     (dict(pool_k=4), B.CKV_EINVAL), (dict(pool_k=65), B.CKV_ENOTSUP), (dict(dtype=7), B.CKV_EINVAL),
     (dict(alpha=1.5), B.CKV_EINVAL), (dict(alpha=-0.1), B.CKV_EINVAL), (dict(eps=-1.0), B.CKV_EINVAL),
     (dict(budget=513), B.CKV_EINVAL), (dict(budget=-1), B.CKV_EINVAL),

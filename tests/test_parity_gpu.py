@@ -59,6 +59,29 @@ def test_small_and_edge_cases(case):
         pu.check_layer_against_oracle(L, wl, out)
 
 
+LONG_WINDOWS = [
+    # (kwargs, flags name, expected attention path bit set for tcgen05)
+    (dict(dtype="bf16", n=1500, w=128, kp=7, budget=200, dh=128, dm=256, Hq=8, Hkv=2), None, True),   # 2 + 2 heads
+    (dict(dtype="bf16", n=2100, w=256, kp=7, budget=300, dh=128, dm=256, Hq=8, Hkv=2), None, True),   # head by head
+    (dict(dtype="bf16", n=700, w=256, kp=5, budget=90, dh=64, dm=128, Hq=3, Hkv=1), None, True),
+    (dict(dtype="bf16", n=900, w=100, kp=7, budget=120, dh=128, dm=256, Hq=4, Hkv=2), None, False),  # CUDA cores
+    (dict(dtype="bf16", n=900, w=256, kp=7, budget=120, dh=128, dm=256, Hq=4, Hkv=2), "simt", False),
+    (dict(dtype="f32", n=600, w=200, kp=5, budget=70, dh=64, dm=128, Hq=4, Hkv=2), None, False),
+    (dict(dtype="f32", n=256, w=256, kp=3, budget=50, dh=64, dm=128, Hq=2, Hkv=2), None, False),      # n == w
+]
+
+
+@pytest.mark.parametrize("case", range(len(LONG_WINDOWS)))
+def test_long_observation_windows(case):
+    # windows beyond 64 rows (the accumulate-over-many-queries setting of the paper's H2O-style comparison)
+    from paper_2502_03805_b200 import binding as B
+    kw, force, tensor_cores = LONG_WINDOWS[case]
+    wl = small_workload(cfg_id=220 + case, **kw)
+    Ls, outs, s = _run(wl, flags=B.CKV_FLAG_FORCE_SIMT if force else 0)
+    assert bool(s.last_path & 1) == tensor_cores
+    pu.check_layer_against_oracle(Ls[0], wl, outs[0])
+
+
 def test_forced_cuda_core_path_agrees_with_tensor_core_path():
     from paper_2502_03805_b200 import binding as B
     wl = small_workload(cfg_id=131, dtype="bf16", n=1300, w=32, kp=7, budget=200, dh=128, dm=512, Hq=8, Hkv=2)
