@@ -46,6 +46,8 @@ def parse_args():
     p.add_argument("--group-sum", action="store_true",
                    help="measure the grouped-query shortcut of step 2 (CKV_FLAG_WO_GROUP_SUM) instead of the headline path")
     p.add_argument("--l2", action="store_true", help="measure the L2-norm variant of step 2 (CKV_NORM_L2, Gram matrix)")
+    p.add_argument("--cta-pairs", action="store_true",
+                   help="projection norm with two CTAs per MMA (CKV_FLAG_CTA_PAIR_MMA) instead of the default kernel")
     p.add_argument("--no-cpu-baseline", action="store_true")
     p.add_argument("--no-e2e", action="store_true")
     return p.parse_args()
@@ -204,6 +206,8 @@ def main():
     t_gen = time.time() - t_gen
 
     flags = B.CKV_FLAG_WO_GROUP_SUM if args.group_sum else 0
+    if args.cta_pairs:
+        flags |= B.CKV_FLAG_CTA_PAIR_MMA
     s = session_for(wl, nb=nb, device=local, want_stage=False, flags=flags, norm=1 if args.l2 else 0)
     stream = torch.cuda.current_stream()
     gemm_ev = []
@@ -271,8 +275,8 @@ def main():
                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                     "peak_source": f"{how} (sustained bf16, kernel timed inside a long step)",
                     "ms_per_launch": gemm_avg, "flops_per_launch": flops, "traffic": None,
-                    "tensor_core_path": bool(path & 2)}
-        if args.cfg == 3 and not args.group_sum and not args.l2 and (path & 2):
+                    "tensor_core_path": bool(path & 2), "cta_pairs": bool(path & 16)}
+        if args.cfg == 3 and not args.group_sum and not args.l2 and (path & 2) and not (path & 16):
             # dram__bytes_read.sum + dram__bytes_write.sum of vnorm_umma_kernel<128> from the ncu capture summarised in
             # profiles/vnorm_umma_cfg3.md: 211.66 MB for 2 layers; every layer touches its own V, W_O and output once,
             # so the traffic of a launch is proportional to the layers it processes

@@ -72,12 +72,15 @@ enum {
   CKV_FLAG_PROTECT_WINDOW = 1u << 3, /* always keep the last w entries (the observation window): their scores are
                                      raised to the largest float32 in both stages, so they fill stage 1 first and
                                      count against the budget                                                   */
-  CKV_FLAG_WO_GROUP_SUM = 1u << 2 /* grouped-query shortcut of step 2: the W^O slices of a KV group are added
+  CKV_FLAG_WO_GROUP_SUM = 1u << 2, /* grouped-query shortcut of step 2: the W^O slices of a KV group are added
                                      (float32, heads ascending, rounded once to the storage type) and each value
                                      row is projected once per KV head.  vnorm then is [nb, Hkv, n] and
                                      c_g = (a_g + eps) * vnorm_g in criticalkv_select.  Hq/Hkv times fewer flops;
                                      not the per-head norm of Algorithm 1 but the norm of the group's summed
                                      projection (the heads of a group share V, so their outputs add in Eq. 2).  */
+  CKV_FLAG_CTA_PAIR_MMA = 1u << 4 /* bf16 projection norm: use the kernel that pairs two CTAs of a cluster per
+                                     MMA (tcgen05 cta_group::2) instead of the default single-CTA kernel.  Same
+                                     results bit for bit; measured slower on B200 for head_dim 128              */
 };
 
 /* Problem descriptor (plain data, copied by every call). */
@@ -248,7 +251,8 @@ CKV_API const char* criticalkv_status_string(int status);
    until the next call on the handle. */
 CKV_API const char* criticalkv_last_cuda_error(criticalkv_handle h);
 /* Which kernels the last criticalkv_score on this handle launched: bit0 tensor-core window attention,
-   bit1 tensor-core projection norm, bit2 CUDA-core window attention, bit3 CUDA-core projection norm. */
+   bit1 tensor-core projection norm, bit2 CUDA-core window attention, bit3 CUDA-core projection norm,
+   bit4 the tensor-core projection norm ran with paired CTAs. */
 CKV_API int criticalkv_last_path(criticalkv_handle h);
 /* Number of kernel launches this handle has issued since it was created. */
 CKV_API int64_t criticalkv_launch_count(criticalkv_handle h);
