@@ -331,15 +331,70 @@ def compress_layer(Qw, K, V, WO, *, kp, budget_mode, budget, alpha=0.5, eps=1e-4
     return out
 
 
-def chunked_compress(chunks, WO, *, kp, w, budgets, alpha=0.5, eps=1e-4, scale=None):
+def compress_layer_ragged(Qw, K_list, V_list, WO, *, kp, budget_mode, budget, alpha=0.5, eps=1e-4, scale=None):
+    """The whole path for one layer whose KV heads hold different numbers of entries (what adaptive budgets leave
+    behind between the chunks of a chunked prefill).  K_list[g], V_list[g]: [n_g, dh]; the observation window of
+    every head is its own last w entries.  Every step is the per-head definition applied to that head's own list;
+    the adaptive allocation ranks the attention scores of all heads' entries together, ties going to the lower
+    (head, entry) pair.
+
+    Returns dict(P [Hq] list of [n_g] arrays, nu likewise, a, c [Hkv] lists of float32 arrays, budgets [Hkv],
+    idx (entry numbers inside each head's own list, packed by head, ascending), offsets [Hkv+1], stage).
+    """
+    Hq, w, dh = Qw.shape
+    Hkv = len(K_list)
+    G = Hq // Hkv
+    if scale is None or scale <= 0:
+        scale = 1.0 / math.sqrt(dh)
+    P, nu = [], []
+    for h in range(Hq):
+        g = h // G
+        P.append(max_pool(window_mean(window_softmax(Qw[h], K_list[g], scale)), kp))
+        nu.append(projection_norm(np.asarray(V_list[g])[None], np.asarray(WO[h])[None])[0])
+    a, c = [], []
+    for g in range(Hkv):
+        ag, cg = group_scores(np.stack(P[g * G:(g + 1) * G]), np.stack(nu[g * G:(g + 1) * G]), G, eps)
+        a.append(ag[0])
+        c.append(cg[0])
+    lens = np.array([x.shape[0] for x in a], dtype=np.int64)
+    if budget_mode == "uniform":
+        budgets = np.full(Hkv, int(budget), dtype=np.int64)
+    elif budget_mode == "adaptive":
+        start = np.concatenate([[0], np.cumsum(lens)])
+        top = stable_topk(np.concatenate(a), int(budget))             # order of the concatenation = (head, entry)
+        head_of = np.searchsorted(start, top, side="right") - 1
+        budgets = np.bincount(head_of, minlength=Hkv).astype(np.int64)
+    else:
+        raise ValueError(budget_mode)
+    if np.any(budgets > lens):
+        raise ValueError("a head's budget exceeds the entries it holds")
+    idx, stage, offsets = [], [], [0]
+    for g in range(Hkv):
+        S1, S2 = two_stage_select(a[g], c[g], int(budgets[g]), alpha)
+        S = np.concatenate([S1, S2])
+        st = np.concatenate([np.ones(S1.size, np.uint8), np.full(S2.size, 2, np.uint8)])
+        order = np.argsort(S, kind="stable")
+        idx.append(S[order])
+        stage.append(st[order])
+        offsets.append(offsets[-1] + S.size)
+    return dict(P=P, nu=nu, a=a, c=c, budgets=budgets, idx=np.concatenate(idx).astype(np.int32),
+                stage=np.concatenate(stage), offsets=np.asarray(offsets, dtype=np.int32))
+
+
+def chunked_compress(chunks, WO, *, kp, w, budgets, alpha=0.5, eps=1e-4, scale=None, budget_mode="uniform"):
     """Chunked prefill with eviction between chunks (the paper's long-context deployment, appendix on chunked
     prefill): for every chunk the cache is [retained entries ; the chunk's K, V], the observation window is the last
-    w queries of the chunk, and the cache is compressed to ``budgets[c]`` entries per KV head (uniform budgets, so
-    every head keeps the same number).  Later chunks therefore see a smaller cache.
+    w queries of the chunk, and the cache is compressed to ``budgets[c]``: entries per KV head with uniform budgets
+    (every head keeps the same number), entries per layer with adaptive budgets (the heads then keep different
+    numbers and the next chunk meets a ragged cache).  Later chunks therefore see a smaller cache.
 
     chunks: list of (Qw [Hq,w,dh], K [Hkv,len,dh], V [Hkv,len,dh]) widened inputs.
-    Returns (K_ret, V_ret [Hkv, B_last, dh], pos [Hkv, B_last] original token positions, history of per-step idx).
+    Returns (K_ret, V_ret, pos, history of per-step idx): uniform budgets give arrays [Hkv, B_last, dh] and
+    [Hkv, B_last] (original token positions) and idx [Hkv, B]; adaptive budgets give per-head lists of arrays
+    and, per step, the list of each head's retained entry numbers.
     """
+    if budget_mode == "adaptive":
+        return _chunked_compress_adaptive(chunks, WO, kp=kp, budgets=budgets, alpha=alpha, eps=eps, scale=scale)
     K_ret = V_ret = pos = None
     seen = 0
     hist = []
@@ -361,6 +416,31 @@ def chunked_compress(chunks, WO, *, kp, w, budgets, alpha=0.5, eps=1e-4, scale=N
         V_ret = np.stack([Vc[g][idx[g]] for g in range(Hkv)])
         pos = np.stack([pc[g][idx[g]] for g in range(Hkv)])
         hist.append(idx)
+    return K_ret, V_ret, pos, hist
+
+
+def _chunked_compress_adaptive(chunks, WO, *, kp, budgets, alpha, eps, scale):
+    K_ret = V_ret = pos = None
+    seen = 0
+    hist = []
+    for c, (Qw, K, V) in enumerate(chunks):
+        Hkv, ln, _ = K.shape
+        new_pos = np.arange(seen, seen + ln, dtype=np.int64)
+        if K_ret is None:
+            Kc, Vc, pc = [K[g] for g in range(Hkv)], [V[g] for g in range(Hkv)], [new_pos] * Hkv
+        else:
+            Kc = [np.concatenate([K_ret[g], K[g]], axis=0) for g in range(Hkv)]
+            Vc = [np.concatenate([V_ret[g], V[g]], axis=0) for g in range(Hkv)]
+            pc = [np.concatenate([pos[g], new_pos]) for g in range(Hkv)]
+        seen += ln
+        out = compress_layer_ragged(Qw, Kc, Vc, WO, kp=kp, budget_mode="adaptive", budget=int(budgets[c]),
+                                    alpha=alpha, eps=eps, scale=scale)
+        off = out["offsets"]
+        kept = [out["idx"][off[g]:off[g + 1]] for g in range(Hkv)]
+        K_ret = [Kc[g][kept[g]] for g in range(Hkv)]
+        V_ret = [Vc[g][kept[g]] for g in range(Hkv)]
+        pos = [pc[g][kept[g]] for g in range(Hkv)]
+        hist.append(kept)
     return K_ret, V_ret, pos, hist
 
 

@@ -571,6 +571,84 @@ def test_chunked_compress_single_chunk_and_positions():
             np.testing.assert_array_equal(krow, src)
 
 
+def _ragged_case(cut=(0, 37), **kw):
+    from gen import make_layer, small_workload
+    wl = small_workload(n=160, w=8, kp=5, cfg_id=72, **kw)
+    L = make_layer(wl)
+    K_list = [L.K[g][cut[g]:] for g in range(wl.Hkv)]
+    V_list = [L.V[g][cut[g]:] for g in range(wl.Hkv)]
+    return wl, L, K_list, V_list
+
+
+@pytest.mark.parametrize("mode,budget", [("uniform", 31), ("adaptive", 70)])
+def test_ragged_compress_with_equal_lengths_is_the_plain_path(mode, budget):
+    wl, L, K_list, V_list = _ragged_case(cut=(0, 0))
+    rag = oc.compress_layer_ragged(L.Qw, K_list, V_list, L.WO, kp=wl.kp, budget_mode=mode, budget=budget)
+    ref = oc.compress_layer(L.Qw, L.K, L.V, L.WO, kp=wl.kp, budget_mode=mode, budget=budget)
+    np.testing.assert_array_equal(rag["idx"], ref["idx"])
+    np.testing.assert_array_equal(rag["offsets"], ref["offsets"])
+    np.testing.assert_array_equal(rag["stage"], ref["stage"])
+    np.testing.assert_array_equal(np.stack(rag["P"]), ref["P"])
+
+
+def test_ragged_compress_treats_every_head_as_its_own_sequence():
+    # a head's scores depend only on its own list: they equal the plain path run on that head alone, and the
+    # adaptive allocation equals a brute-force ranking of all (score, head, entry) triples
+    wl, L, K_list, V_list = _ragged_case(cut=(0, 37))
+    B = 90
+    rag = oc.compress_layer_ragged(L.Qw, K_list, V_list, L.WO, kp=wl.kp, budget_mode="adaptive", budget=B)
+    G = wl.G
+    for g in range(wl.Hkv):
+        alone = oc.compress_layer(L.Qw[g * G:(g + 1) * G], K_list[g][None], V_list[g][None], L.WO[g * G:(g + 1) * G],
+                                  kp=wl.kp, budget_mode="uniform", budget=int(rag["budgets"][g]))
+        np.testing.assert_array_equal(alone["a"][0], rag["a"][g])
+        np.testing.assert_array_equal(alone["c"][0], rag["c"][g])
+        np.testing.assert_array_equal(alone["idx"], rag["idx"][rag["offsets"][g]:rag["offsets"][g + 1]])
+    triples = sorted(((-float(v), g, i) for g in range(wl.Hkv) for i, v in enumerate(rag["a"][g])))[:B]
+    counts = np.bincount([t[1] for t in triples], minlength=wl.Hkv)
+    np.testing.assert_array_equal(counts, rag["budgets"])
+    assert rag["budgets"].sum() == B and np.all(rag["budgets"] <= [k.shape[0] for k in K_list])
+
+
+def test_ragged_compress_equals_left_padded_selection_with_excluded_padding():
+    # the layout the CUDA path uses: heads right-aligned in a common length, padding scored below every real entry
+    wl, L, K_list, V_list = _ragged_case(cut=(0, 37))
+    cut = (0, 37)
+    rag = oc.compress_layer_ragged(L.Qw, K_list, V_list, L.WO, kp=wl.kp, budget_mode="adaptive", budget=90)
+    n = wl.n
+    a = np.full((wl.Hkv, n), -1.0, np.float32)
+    c = np.full((wl.Hkv, n), -1.0, np.float32)
+    for g in range(wl.Hkv):
+        a[g, cut[g]:], c[g, cut[g]:] = rag["a"][g], rag["c"][g]
+    budgets = oc.allocate_budgets(a, "adaptive", 90)
+    np.testing.assert_array_equal(budgets, rag["budgets"])
+    for g in range(wl.Hkv):
+        S1, S2 = oc.two_stage_select(a[g], c[g], int(budgets[g]), 0.5)
+        got = np.sort(np.concatenate([S1, S2])) - cut[g]
+        np.testing.assert_array_equal(got, rag["idx"][rag["offsets"][g]:rag["offsets"][g + 1]])
+
+
+def test_chunked_compress_adaptive_budgets_leave_a_ragged_cache():
+    from gen import make_layer, small_workload
+    wl = small_workload(n=120, w=8, kp=5, budget=30, cfg_id=73)
+    L = make_layer(wl)
+    L2 = make_layer(wl.with_(n=60), 1)
+    chunks = [(L.Qw, L.K, L.V), (L2.Qw, L2.K, L2.V)]
+    K1, V1, pos1, hist1 = oc.chunked_compress(chunks[:1], L.WO, kp=wl.kp, w=wl.w, budgets=[70], budget_mode="adaptive")
+    ref = oc.compress_layer(L.Qw, L.K, L.V, L.WO, kp=wl.kp, budget_mode="adaptive", budget=70)
+    for g in range(wl.Hkv):
+        np.testing.assert_array_equal(pos1[g], ref["idx"][ref["offsets"][g]:ref["offsets"][g + 1]])
+    K2, V2, pos2, hist2 = oc.chunked_compress(chunks, L.WO, kp=wl.kp, w=wl.w, budgets=[70, 90],
+                                              budget_mode="adaptive")
+    assert sum(p.size for p in pos2) == 90
+    for g in range(wl.Hkv):
+        assert np.all(np.diff(pos2[g]) > 0) and pos2[g].max() < 180
+        assert set(pos2[g][pos2[g] < 120].tolist()) <= set(pos1[g].tolist())
+        for p, krow, vrow in zip(pos2[g], K2[g], V2[g]):
+            np.testing.assert_array_equal(krow, L.K[g][p] if p < 120 else L2.K[g][p - 120])
+            np.testing.assert_array_equal(vrow, L.V[g][p] if p < 120 else L2.V[g][p - 120])
+
+
 def test_compress_layer_end_to_end_small():
     from gen import make_layer, small_workload
     wl = small_workload(n=96, w=8, kp=5, budget=20)
