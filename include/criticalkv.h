@@ -110,6 +110,14 @@ typedef struct {
                             floor(adaptive_floor * budget / Hkv) entries, the rest of the budget goes to the
                             flattened top-k, and a head's budget is capped at n.  0 in the paper's settings.   */
   uint32_t reserved2;    /* must be 0                                                                   */
+  const int32_t* valid_from; /* NULL, or device int32 [nb,Hkv]: KV head g of slice b holds its entries right-aligned,
+                            rows i < valid_from[b,g] of K and V are padding (0 <= valid_from <= n - w).  Padding
+                            is invisible to the window queries, gets attn = 0 and the scores a = c = -1, below
+                            every real entry, so it is selected only if a head's budget exceeds its n -
+                            valid_from real entries (the caller's to avoid; adaptive allocation never does while
+                            budget <= number of real entries).  This is the ragged cache that adaptive budgets
+                            leave between the chunks of a chunked prefill.  Not accepted by
+                            criticalkv_compress_host and criticalkv_diagnose.                              */
 } criticalkv_desc;
 
 /* Create / destroy a handle bound to CUDA device `device`.  create allocates one device status word. */

@@ -38,7 +38,7 @@ class criticalkv_desc(C.Structure):
                 ("budget_mode", C.c_int32), ("norm", C.c_int32), ("budget", C.c_int64),
                 ("flags", C.c_uint32), ("reserved", C.c_uint32),
                 ("q_stride", C.c_int64 * 3), ("k_stride", C.c_int64 * 3), ("v_stride", C.c_int64 * 3),
-                ("adaptive_floor", C.c_float), ("reserved2", C.c_uint32)]
+                ("adaptive_floor", C.c_float), ("reserved2", C.c_uint32), ("valid_from", C.c_void_p)]
 
 
 class CriticalKVError(RuntimeError):
@@ -119,7 +119,9 @@ def status_string(status: int) -> str:
 
 def make_desc(*, nb, Hq, Hkv, dh, dm, n, w, pool_k, dtype, budget_mode, budget, alpha=0.5, eps=1e-4, scale=0.0,
               flags=0, norm=CKV_NORM_L1, q_stride=(0, 0, 0), k_stride=(0, 0, 0), v_stride=(0, 0, 0),
-              adaptive_floor=0.0):
+              adaptive_floor=0.0, valid_from=None):
+    """valid_from: device int32 tensor [nb, Hkv] (or an address) for right-aligned ragged heads; the caller keeps it
+    alive while the descriptor is in use."""
     d = criticalkv_desc()
     d.nb, d.Hq, d.Hkv, d.dh, d.dm, d.n, d.w, d.pool_k = nb, Hq, Hkv, dh, dm, n, w, pool_k
     d.dtype = {"f32": CKV_F32, "bf16": CKV_BF16}.get(dtype, dtype)
@@ -131,6 +133,8 @@ def make_desc(*, nb, Hq, Hkv, dh, dm, n, w, pool_k, dtype, budget_mode, budget, 
     d.k_stride[:] = k_stride
     d.v_stride[:] = v_stride
     d.adaptive_floor, d.reserved2 = adaptive_floor, 0
+    d.valid_from = None if valid_from is None else (valid_from if isinstance(valid_from, int)
+                                                    else valid_from.data_ptr())
     return d
 
 

@@ -98,6 +98,8 @@ int resolve(const criticalkv_desc* d, Dims* o) {
     if (o->qs[i] % vec || o->ks[i] % vec || o->vs[i] % vec) return CKV_EALIGN;
   }
   if (o->qs[2] < d->dh || o->ks[2] < d->dh || o->vs[2] < d->dh) return CKV_EINVAL;
+  if (reinterpret_cast<uintptr_t>(d->valid_from) & 3u) return CKV_EALIGN;
+  o->valid_from = d->valid_from;
   return CKV_OK;
 }
 
@@ -448,6 +450,7 @@ int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc* d, cons
   if (rc != CKV_OK) return rc;
   if (!Qw || !K || !V || !WO || !idx || !offsets || !K_out || !V_out || !staging) return CKV_EINVAL;
   if (dd.budget_mode == CKV_BUDGET_GIVEN && !budgets_in) return CKV_EINVAL;
+  if (d->valid_from) return CKV_ENOTSUP;   // the per-head offsets would have to be host memory here
   for (int i = 0; i < 3; ++i)
     if (d->q_stride[i] || d->k_stride[i] || d->v_stride[i]) return CKV_ENOTSUP;  // host arrays must be dense
   if (reinterpret_cast<uintptr_t>(staging) & 255u) return CKV_EALIGN;
@@ -544,6 +547,7 @@ int criticalkv_diagnose(criticalkv_handle h, const criticalkv_desc* d, const voi
   int rc = resolve(d, &dd);
   if (rc != CKV_OK) return rc;
   if (dd.group_sum) return CKV_ENOTSUP;  // the bounds are stated with per-head norms
+  if (dd.valid_from) return CKV_ENOTSUP;
   if (dd.w > 64) return CKV_ENOTSUP;     // the diagnostics kernel keeps a window's rows in registers
   if (!Qw || !K || !V || !WO || !vnorm || !idx || !offsets || !stage || !diag || !ws) return CKV_EINVAL;
   if (!aligned16(Qw) || !aligned16(K) || !aligned16(V) || !aligned16(WO) || !aligned16(vnorm) || !aligned16(diag) ||

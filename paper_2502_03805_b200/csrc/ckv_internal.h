@@ -21,6 +21,7 @@ struct Dims {
   int norm;           // criticalkv_norm
   long long floor_b;  // guaranteed entries per KV head (adaptive budgets)
   long long qs[3], ks[3], vs[3];  // element strides: nb, head, row
+  const int32_t* valid_from;      // device [nb, Hkv] or null: first real row of every KV head (rows before it are padding)
 };
 
 // Keys of the window-attention kernels are processed in chunks of this many tokens (one CTA each).

@@ -26,7 +26,8 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 __global__ void group_reduce_kernel(const float* __restrict__ attn, const float* __restrict__ vnorm,
                                     float* __restrict__ a, float* __restrict__ c, int Hq, int Hkv, int G, int n,
-                                    float eps, int group_sum, int protect_from) {
+                                    float eps, int group_sum, int protect_from,
+                                    const int32_t* __restrict__ valid_from) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   const int g = blockIdx.y, b = blockIdx.z;
@@ -52,6 +53,8 @@ __global__ void group_reduce_kernel(const float* __restrict__ attn, const float*
     cv = __fdiv_rn(sc, Gf);
   }
   if (i >= protect_from) av = cv = 3.402823466e+38f;  // protected observation window: largest float32
+  // padding in front of a right-aligned head: below every real score (those are >= 0), so it is taken last
+  if (valid_from != nullptr && i < valid_from[b * Hkv + g]) av = cv = -1.0f;
   if (av == 0.f) av = 0.f;  // -0 and +0 must order alike
   if (cv == 0.f) cv = 0.f;
   const long long o = ((long long)b * Hkv + g) * n + i;
@@ -434,7 +437,7 @@ cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* v
                                 cudaStream_t st, int* launches) {
   dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
   group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, a, c, d.Hq, d.Hkv, d.G, d.n, d.eps, d.group_sum,
-                                             d.protect_window ? d.n - d.w : d.n);
+                                             d.protect_window ? d.n - d.w : d.n, d.valid_from);
   *launches += 1;
   return cudaGetLastError();
 }

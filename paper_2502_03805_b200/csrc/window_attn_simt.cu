@@ -27,6 +27,7 @@ struct AttnArgs {
   float* rowstat;
   float* abar;
   int Hq, G, n, w, nchunks;
+  const int32_t* valid_from;   // [nb, Hkv] or null: first real key of every KV head
   float scale;
   long long qs[3], ks[3];
 };
@@ -55,6 +56,7 @@ __global__ void __launch_bounds__(kThreads) attn_pass_kernel(AttnArgs a) {
   const long long row = (long long)(b * a.Hq + h) * a.w;
   const bool in_range = i < a.n;
   const int first_pos = a.n - a.w;  // sequence position of window row 0
+  const int vf = a.valid_from ? a.valid_from[b * (a.Hq / a.G) + g] : 0;   // keys before vf are padding
   float s = 0.f;                    // second pass: sum of the normalised weights over the window rows
   // the window is walked in blocks of WT rows (one block unless w > 64)
   for (int j0 = 0; j0 < a.w; j0 += WT) {
@@ -76,7 +78,7 @@ __global__ void __launch_bounds__(kThreads) attn_pass_kernel(AttnArgs a) {
     }
 #pragma unroll
     for (int j = 0; j < WT; ++j) {
-      const bool visible = in_range && j < wb && i <= first_pos + j0 + j;
+      const bool visible = in_range && j < wb && i <= first_pos + j0 + j && i >= vf;
       acc[j] = visible ? acc[j] * a.scale : -INFINITY;
     }
 
@@ -236,6 +238,7 @@ static AttnArgs make_attn_args(const Dims& d, const void* Qw, const void* K, con
   a.part_m = ws.part_m; a.part_l = ws.part_l; a.rowstat = ws.rowstat; a.abar = ws.abar;
   a.Hq = d.Hq; a.G = d.G; a.n = d.n; a.w = d.w;
   a.nchunks = (d.n + kAttnChunk - 1) / kAttnChunk;
+  a.valid_from = d.valid_from;
   a.scale = d.scale;
   for (int i = 0; i < 3; ++i) { a.qs[i] = d.qs[i]; a.ks[i] = d.ks[i]; }
   return a;
@@ -252,13 +255,7 @@ cudaError_t launch_window_stats_simt(const Dims& d, const void* Qw, const void* 
 
 cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K, float* attn,
                                     const ScoreWorkspace& ws, cudaStream_t st, int* launches) {
-  AttnArgs a;
-  a.Qw = Qw; a.K = K;
-  a.part_m = ws.part_m; a.part_l = ws.part_l; a.rowstat = ws.rowstat; a.abar = ws.abar;
-  a.Hq = d.Hq; a.G = d.G; a.n = d.n; a.w = d.w;
-  a.nchunks = (d.n + kAttnChunk - 1) / kAttnChunk;
-  a.scale = d.scale;
-  for (int i = 0; i < 3; ++i) { a.qs[i] = d.qs[i]; a.ks[i] = d.ks[i]; }
+  const AttnArgs a = make_attn_args(d, Qw, K, ws);
   if (d.dtype == CKV_F32) {
     return d.dh == 64 ? run_w<float, 64>(d, a, attn, st, launches) : run_w<float, 128>(d, a, attn, st, launches);
   }

@@ -45,6 +45,7 @@ struct AttnUmmaArgs {
   float* part_l;
   const float* rowstat;
   float* abar;
+  const int32_t* valid_from;   // [nb, Hkv] or null: first real key of every KV head (keys before it are padding)
   int* status;
   int Hq, Hkv, G, n, nb;
   int Gi;              // query heads per work item: the largest divisor of G with Gi * w <= 384
@@ -289,13 +290,15 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
         }
       }
       const float* st = stats + qb * a.rows;
+      const int vf = a.valid_from ? a.valid_from[w.b * a.Hkv + w.g] : 0;
       float rm[kMaxRowBlocks], rl[kMaxRowBlocks];
 #pragma unroll
       for (int rb = 0; rb < kMaxRowBlocks; ++rb) { rm[rb] = -INFINITY; rl[rb] = 0.f; }
 
       for (int kt = w.t0; kt < w.t1 && !failed; ++kt) {
         const int key0 = kt * kKeyTile;
-        const bool tail = key0 + kKeyTile - 1 > first_pos;  // some (key, row) pair of this tile is masked
+        // some (key, row) pair of this tile is masked: causally (last tiles) or as padding (first tiles)
+        const bool tail = key0 + kKeyTile - 1 > first_pos || key0 < vf;
 #pragma unroll 1
         for (int sub = 0; sub < nsub; ++sub, ++t) {
           if ((t & 1u) != set) continue;
@@ -323,7 +326,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                 for (int q = 0; q < CW / 32; ++q)
 #pragma unroll
                   for (int e = 0; e < 32; ++e)
-                    if (key0 + c0 + q * 32 + e > lim) v[q][e] = -INFINITY;
+                    if (key0 + c0 + q * 32 + e > lim || key0 + c0 + q * 32 + e < vf) v[q][e] = -INFINITY;
               }
               float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
 #pragma unroll
@@ -398,7 +401,8 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
                     a3 += ex2_approx(fmaf(v[(j + 3) / 16][(j + 3) % 16], a.c, bz.w));
                   }
                 } else {
-                  const int jmin = i - first_pos - jc;              // rows jc + j with j < jmin do not see key i
+                  // rows jc + j with j < jmin do not see key i; a padding key is seen by no row
+                  const int jmin = i >= vf ? i - first_pos - jc : W;
 #pragma unroll
                   for (int j = 0; j < JC; j += 4) {
                     const float4 bz = sr[j / 4];
@@ -488,6 +492,7 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
 
   AttnUmmaArgs a;
   a.part_m = ws.part_m; a.part_l = ws.part_l; a.rowstat = ws.rowstat; a.abar = ws.abar; a.status = status_word;
+  a.valid_from = d.valid_from;
   a.Hq = d.Hq; a.Hkv = d.Hkv; a.G = d.G; a.n = d.n; a.nb = d.nb;
   a.Gi = Gi;
   a.subgroups = d.G / Gi;

@@ -308,6 +308,99 @@ def test_chunked_prefill_matches_oracle(dtype):
     np.testing.assert_array_equal(Vg, Vr)
 
 
+def _padded_selection_reference(rag, cuts, n):
+    """The oracle's ragged result in the coordinates of the right-aligned layout (padding scored -1)."""
+    Hkv = len(cuts)
+    a = np.full((Hkv, n), -1.0, np.float32)
+    c = np.full((Hkv, n), -1.0, np.float32)
+    idx = rag["idx"].copy()
+    for g in range(Hkv):
+        a[g, cuts[g]:], c[g, cuts[g]:] = rag["a"][g], rag["c"][g]
+        idx[rag["offsets"][g]:rag["offsets"][g + 1]] += cuts[g]
+    return dict(a=a, c=c, budgets=rag["budgets"], idx=idx, offsets=rag["offsets"], stage=rag["stage"])
+
+
+def _check_ragged_call(Qw, K_lists, V_lists, WO, cuts, n, wl, out, budget_mode, budget):
+    """out: host arrays of one GPU call on right-aligned heads; K_lists / V_lists: each head's real rows (widened)."""
+    rag = oc.compress_layer_ragged(Qw, K_lists, V_lists, WO, kp=wl.kp, budget_mode=budget_mode, budget=budget,
+                                   alpha=wl.alpha, eps=wl.eps)
+    for h in range(wl.Hq):
+        g = h // wl.G
+        pu.assert_scores_close(out["attn"][h, cuts[g]:], rag["P"][h], f"attn head {h}")
+        pu.assert_scores_close(out["vnorm"][h, cuts[g]:], rag["nu"][h], f"vnorm head {h}")
+    ref = _padded_selection_reference(rag, cuts, n)
+    rep = pu.compare_selection(ref, out["idx"], out["offsets"], out.get("stage"), n=n, alpha=wl.alpha,
+                               budget_mode=budget_mode, budget=budget)
+    for g in range(wl.Hkv):
+        seg = out["idx"][out["offsets"][g]:out["offsets"][g + 1]]
+        assert seg.size == 0 or seg.min() >= cuts[g], f"head {g}: a padding row was selected"
+    return rep
+
+
+@pytest.mark.parametrize("dtype,mode,budget", [("bf16", "adaptive", 900), ("bf16", "uniform", 300),
+                                               ("f32", "adaptive", 700)])
+def test_right_aligned_ragged_heads_match_the_per_head_oracle(dtype, mode, budget):
+    # heads of different lengths in one call: head g's real rows start at cuts[g]; the rows before are padding filled
+    # with large values that would dominate the softmax if they were visible
+    from gen import f32_to_bf16_bits
+    from gpu_util import run_layers
+    wl = small_workload(cfg_id=230, dtype=dtype, n=1000, w=32, kp=7, budget_mode=mode, budget=budget,
+                        dh=128 if dtype == "bf16" else 64, dm=256, Hq=8, Hkv=4)
+    L = make_layer(wl, 0)
+    cuts = [0, 300, 129, 511]            # a fully padded tile plus a straddling one, a one-key overhang, ...
+    fill = f32_to_bf16_bits(np.float32(30.0)) if dtype == "bf16" else np.float32(30.0)
+    for g in range(wl.Hkv):
+        L.K_store[g, :cuts[g]] = fill
+        L.V_store[g, :cuts[g]] = fill
+    vf = torch.tensor([cuts], dtype=torch.int32, device="cuda")
+    outs, s = run_layers([L], wl, valid_from=vf)
+    K_lists = [L.K[g][cuts[g]:] for g in range(wl.Hkv)]
+    V_lists = [L.V[g][cuts[g]:] for g in range(wl.Hkv)]
+    _check_ragged_call(L.Qw, K_lists, V_lists, L.WO, cuts, wl.n, wl, outs[0], mode, budget)
+    pu.assert_compaction_exact(L.K_store, L.V_store, outs[0]["idx"], outs[0]["offsets"], outs[0]["K_out"],
+                               outs[0]["V_out"])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_chunked_prefill_with_adaptive_budgets_matches_oracle_step_by_step(dtype):
+    # adaptive budgets leave the heads with different numbers of entries; every step is checked against the oracle run
+    # on the cache the GPU path holds at that point, and the carried rows and positions against the step's own indices
+    from gen import bf16_bits_to_f32
+    from paper_2502_03805_b200 import ChunkedPrefillCompressor, to_device, to_host
+    base = small_workload(cfg_id=181, dtype=dtype, Hq=4, Hkv=2, dh=128 if dtype == "bf16" else 64, dm=256, n=600,
+                          w=16, kp=5, budget_mode="adaptive", budget=500)
+    lens, budgets = [600, 500, 300], [500, 700, 600]
+    Ls = [make_layer(base.with_(n=ln), c) for c, ln in enumerate(lens)]
+    widen = (lambda x: bf16_bits_to_f32(x).astype(np.float64)) if dtype == "bf16" else (lambda x: x.astype(np.float64))
+    cp = ChunkedPrefillCompressor(Hq=base.Hq, Hkv=base.Hkv, dh=base.dh, dm=base.dm, w=base.w, pool_k=base.kp,
+                                  dtype=dtype, budget_mode="adaptive")
+    dWO = to_device(Ls[0].WO_store, dtype)
+    seen = 0
+    for L, ln, b in zip(Ls, lens, budgets):
+        prev = None if cp.K is None else ([widen(to_host(k)) for k in cp.K], [widen(to_host(v)) for v in cp.V],
+                                          [to_host(p) for p in cp.pos])
+        s = cp.step(to_device(L.Qw_store, dtype), to_device(L.K_store, dtype), to_device(L.V_store, dtype), dWO, b)
+        torch.cuda.synchronize()
+        assert s.device_status() == 0
+        kept = [0] * base.Hkv if prev is None else [k.shape[0] for k in prev[0]]
+        n_max = cp.last["n"]
+        cuts = [n_max - ln - k for k in kept]
+        K_lists = [L.K[g] if prev is None else np.concatenate([prev[0][g], L.K[g]]) for g in range(base.Hkv)]
+        V_lists = [L.V[g] if prev is None else np.concatenate([prev[1][g], L.V[g]]) for g in range(base.Hkv)]
+        out = dict(attn=to_host(s.attn[0]), vnorm=to_host(s.vnorm[0]), idx=to_host(s.idx[0]),
+                   offsets=to_host(s.offsets[0]), stage=to_host(s.stage[0]))
+        _check_ragged_call(L.Qw, K_lists, V_lists, Ls[0].WO, cuts, n_max, base, out, "adaptive", b)
+        new_pos = np.arange(seen, seen + ln)
+        for g in range(base.Hkv):
+            local = out["idx"][out["offsets"][g]:out["offsets"][g + 1]] - cuts[g]
+            pc = new_pos if prev is None else np.concatenate([prev[2][g], new_pos])
+            np.testing.assert_array_equal(to_host(cp.pos[g]), pc[local])
+            np.testing.assert_array_equal(widen(to_host(cp.K[g])), K_lists[g][local])
+            np.testing.assert_array_equal(widen(to_host(cp.V[g])), V_lists[g][local])
+        seen += ln
+    assert sum(int(p.shape[0]) for p in cp.pos) == budgets[-1]
+
+
 @pytest.mark.parametrize("kw", [
     dict(dtype="f32", n=500, w=16, kp=5, budget=120, dh=64, dm=192, Hq=4, Hkv=2),
     dict(dtype="bf16", n=1100, w=32, kp=7, budget=300, dh=128, dm=256, Hq=4, Hkv=2),
