@@ -538,6 +538,55 @@ def test_config3_two_layers_adaptive_parity():
         print("config3 layer", L.layer, rep)
 
 
+def test_config3_all_layers_in_one_call_as_benchmarked():
+    # the launch configuration the benchmark times: all 32 layers in one call (nb = 32).  Every layer is checked by
+    # properties that hold at any size (budgets, ordering, the selection rule applied to the GPU's own float32 scores,
+    # bit-exact gather) and by sampled outputs the oracle computes one by one (one query head's attention row and
+    # 256 projection norms per layer).
+    from paper_2502_03805_b200 import session_for, to_device, to_host
+    wl = config(3)
+    nb, n, G = wl.layers, wl.n, wl.G
+    bf = torch.bfloat16
+    Qw = torch.empty((nb, wl.Hq, wl.w, wl.dh), dtype=bf, device="cuda")
+    K = torch.empty((nb, wl.Hkv, n, wl.dh), dtype=bf, device="cuda")
+    V = torch.empty_like(K)
+    WO = torch.empty((nb, wl.Hq, wl.dh, wl.dm), dtype=bf, device="cuda")
+    rng = np.random.default_rng(33)
+    scale = wl.scale
+    expected = []
+    for l in range(nb):
+        L = make_layer(wl, l)
+        for dst, name in ((Qw, "Qw_store"), (K, "K_store"), (V, "V_store"), (WO, "WO_store")):
+            dst[l].copy_(to_device(getattr(L, name), "bf16"))
+        h = int(rng.integers(wl.Hq))
+        rows = np.sort(rng.choice(n, 256, replace=False))
+        P_h = oc.max_pool(oc.window_mean(oc.window_softmax(L.Qw[h], L.K[h // G], scale)), wl.kp)
+        nu_h = oc.projection_norm(L.V[h // G][None], L.WO[h][None], rows=rows)[0]
+        expected.append((h, rows, P_h, nu_h))
+        del L
+    s = session_for(wl, nb=nb)
+    s.compress(Qw, K, V, WO)
+    torch.cuda.synchronize()
+    assert s.device_status() == 0 and (s.last_path & 15) == 3
+    K16, V16 = K.view(torch.int16), V.view(torch.int16)
+    Ko16, Vo16 = s.K_out.view(torch.int16), s.V_out.view(torch.int16)
+    for l in range(nb):
+        h, rows, P_h, nu_h = expected[l]
+        attn, vnorm = to_host(s.attn[l]), to_host(s.vnorm[l])
+        pu.assert_scores_close(attn[h], P_h, f"layer {l} attn head {h}")
+        pu.assert_scores_close(vnorm[h, rows], nu_h, f"layer {l} vnorm head {h} (sampled rows)")
+        ref = oc.select(attn, vnorm, G=G, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps)
+        off = to_host(s.offsets[l])
+        np.testing.assert_array_equal(off, ref["offsets"])
+        assert off[-1] == wl.budget
+        np.testing.assert_array_equal(to_host(s.idx[l])[: off[-1]], ref["idx"])
+        np.testing.assert_array_equal(to_host(s.stage[l])[: off[-1]], ref["stage"])
+        for g in range(wl.Hkv):
+            sel = s.idx[l, off[g]:off[g + 1]].long()
+            assert torch.equal(K16[l, g][sel], Ko16[l, off[g]:off[g + 1]])
+            assert torch.equal(V16[l, g][sel], Vo16[l, off[g]:off[g + 1]])
+
+
 @pytest.mark.parametrize("mode", ["uniform", "adaptive"])
 def test_config4_one_layer_sampled(mode):
     # n = 131072: attention compared in full, the projection norm on 4096 sampled rows per head, and the selection
