@@ -253,6 +253,24 @@ def main():
     gemm_ms = [a.elapsed_time(b) for a, b in gemm_ev]
     path = s.last_path
 
+    # ---- per-stage device times, taken after the timed region (three more steps with events between the stages) ----
+    stage_ms = {"window_attention": [], "projection_norm": [], "select": [], "compact": []}
+    for _ in range(3):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        ev[0].record(stream)
+        B.criticalkv_score(s.handle, s.desc, Qw, K, None, None, s.attn, None, s.ws, stream=stream)
+        ev[1].record(stream)
+        B.criticalkv_score(s.handle, s.desc, None, None, V, WO, None, s.vnorm, s.ws, stream=stream)
+        ev[2].record(stream)
+        s.select(stream=stream)
+        ev[3].record(stream)
+        s.compact(K, V, stream=stream)
+        ev[4].record(stream)
+        torch.cuda.synchronize()
+        for i, k in enumerate(stage_ms):
+            stage_ms[k].append(ev[i].elapsed_time(ev[i + 1]))
+    stage_ms = {k: sorted(v)[1] for k, v in stage_ms.items()}
+
     # ---- end to end: host buffers, copies inside the timed region, layer by layer on two streams ----
     e2e = None
     if not args.no_e2e:
@@ -284,6 +302,16 @@ def main():
             roofline["traffic_unit"] = "bytes per launch (ncu, 2-layer capture scaled by layers)"
             roofline["algorithmic_bytes"] = (2.0 * wl.Hkv * wl.n * wl.dh + 2.0 * wl.Hq * wl.dh * wl.dm +
                                              4.0 * wl.Hq * wl.n) * nb
+        # the memory-bound stages against the measured copy bandwidth (algorithmic bytes: K once, attn out; the
+        # retained rows of K and V read and written once)
+        hbm = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+        es = 2 if wl.dtype == "bf16" else 4
+        attn_bytes = (wl.Hkv * wl.n * wl.dh * es + wl.Hq * wl.w * wl.dh * es + 4.0 * wl.Hq * wl.n) * nb
+        compact_bytes = (4.0 * wl.btot * wl.dh * es + 4.0 * wl.btot) * nb
+        stages = {k: {"ms": v} for k, v in stage_ms.items()}
+        for k, nbytes in (("window_attention", attn_bytes), ("compact", compact_bytes)):
+            gbs = nbytes / (stage_ms[k] * 1e-3) / 1e9
+            stages[k].update({"bound": "hbm", "achieved_gbs": gbs, "peak_gbs": hbm, "frac": gbs / hbm})
         cpu = None
         if not args.no_cpu_baseline:
             entries, dt, cores = oracle_sample(wl, 0)
@@ -300,6 +328,7 @@ def main():
                            "l2": "inputs of one step (5.4 GB) exceed L2; layers are distinct buffers",
                            "ms_per_32_layer_compression": ms_per_step * 32.0 / nb},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
+                "stages": stages,
                 "cpu_baseline": cpu, "input_generation_s": round(t_gen, 1)}
         print(json.dumps(line), flush=True)
     if world > 1:
