@@ -82,6 +82,35 @@ def test_long_observation_windows(case):
     pu.check_layer_against_oracle(Ls[0], wl, outs[0])
 
 
+def _random_shape(seed):
+    r = np.random.default_rng(1000 + seed)
+    dtype = "bf16" if seed % 3 else "f32"
+    Hkv = int(r.choice([1, 2, 3, 4]))
+    G = int(r.choice([1, 2, 3, 4, 5, 8]))
+    dh = int(r.choice([64, 128]))
+    w = int(r.choice([1, 3, 8, 16, 32, 64])) if dtype == "f32" else int(r.choice([16, 32, 64, 7, 48]))
+    n = int(r.integers(max(w, 2), 2600))
+    dm = 8 * int(r.integers(1, 90))
+    kp = int(r.choice([1, 3, 5, 7, 9, 15]))
+    mode = str(r.choice(["uniform", "adaptive"]))
+    frac = float(r.choice([0.0, 0.05, 0.2, 0.5, 1.0]))
+    budget = int(frac * n) if mode == "uniform" else int(frac * n * Hkv)
+    alpha = float(r.choice([0.0, 0.25, 0.5, 0.75, 1.0]))
+    return dict(dtype=dtype, Hq=Hkv * G, Hkv=Hkv, dh=dh, dm=dm, n=n, w=w, kp=kp, budget_mode=mode, budget=budget,
+                alpha=alpha)
+
+
+@pytest.mark.parametrize("seed", range(64))
+def test_random_shapes_against_oracle(seed):
+    # seeded draw over group sizes, head counts, window and pool sizes, ragged n and d_model, budgets from nothing to
+    # everything and the stage split: whatever kernels the dispatch picks must agree with the oracle
+    kw = _random_shape(seed)
+    wl = small_workload(cfg_id=300 + seed, **kw)
+    Ls, outs, s = _run(wl)
+    assert s.device_status() == 0
+    pu.check_layer_against_oracle(Ls[0], wl, outs[0])
+
+
 def test_forced_cuda_core_path_agrees_with_tensor_core_path():
     from paper_2502_03805_b200 import binding as B
     wl = small_workload(cfg_id=131, dtype="bf16", n=1300, w=32, kp=7, budget=200, dh=128, dm=512, Hq=8, Hkv=2)
