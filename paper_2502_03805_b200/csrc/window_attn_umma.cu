@@ -11,6 +11,10 @@
 //                      window rows of each head straight from its tensor-memory lane: the window mean comes out
 //                      without any cross-lane traffic and is written coalesced along the sequence.
 // Max-pooling runs afterwards in the shared pooling kernel.
+// Windows of 128 or 256 rows: a work item covers only as many query heads of the group as fit 384 query rows (two
+// heads, or one), the parts of a group stream the KV head's keys one after another, and sweep 2 reads an accumulator
+// in chunks of 64 columns.  Right-aligned ragged heads (valid_from): keys before a head's first real row are masked
+// like the causally invisible ones.
 //
 // Persistent kernel, one CTA per SM: warp 0 streams K tiles (and the group's Q rows, once per work item) with TMA,
 // warp 1 issues the MMAs, warps 2-9 are two sets of four softmax warps that take alternating accumulators (two

@@ -39,7 +39,7 @@ SMALL = [
     dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=0.25),
     dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=1.0),
     dict(dtype="f32", n=400, w=16, kp=5, budget=60, alpha=0.0),
-    # shapes the tensor-core kernels take (w in {16, 32, 64}), with ragged last tiles and short last work items
+    # shapes the tensor-core kernels take, with ragged last tiles and short last work items
     dict(dtype="bf16", n=700, w=32, kp=7, budget=90, dh=128, dm=384, Hq=8, Hkv=2),
     dict(dtype="bf16", n=3000, w=64, kp=7, budget=250, dh=128, dm=640, Hq=10, Hkv=2),    # 320 query rows per group
     dict(dtype="bf16", n=1000, w=16, kp=5, budget=77, dh=64, dm=192, Hq=4, Hkv=2),
