@@ -271,6 +271,28 @@ def main():
             stage_ms[k].append(ev[i].elapsed_time(ev[i + 1]))
     stage_ms = {k: sorted(v)[1] for k, v in stage_ms.items()}
 
+    # ---- the same step captured once in a CUDA graph and replayed (no host launches between the nine kernels) ----
+    graph_ms = None
+    if world == 1:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(side):
+            graph.capture_begin()
+            B.criticalkv_score(s.handle, s.desc, Qw, K, V, WO, s.attn, s.vnorm, s.ws, stream=side)
+            s.select(stream=side)
+            s.compact(K, V, stream=side)
+            graph.capture_end()
+            for _ in range(2):
+                graph.replay()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(side)
+            for _ in range(args.steps):
+                graph.replay()
+            g1.record(side)
+        torch.cuda.synchronize()
+        graph_ms = g0.elapsed_time(g1) / args.steps
+        assert s.device_status() == 0
+
     # ---- end to end: host buffers, copies inside the timed region, layer by layer on two streams ----
     e2e = None
     if not args.no_e2e:
@@ -329,6 +351,9 @@ def main():
                            "ms_per_32_layer_compression": ms_per_step * 32.0 / nb},
                 "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
                 "stages": stages,
+                "graph_replay": None if graph_ms is None else {
+                    "ms_per_step": graph_ms, "value": nb * wl.Hkv * wl.n / (graph_ms * 1e-3), "unit": UNIT,
+                    "how": "the step captured once in a CUDA graph, replayed back to back after the timed region"},
                 "cpu_baseline": cpu, "input_generation_s": round(t_gen, 1)}
         print(json.dumps(line), flush=True)
     if world > 1:

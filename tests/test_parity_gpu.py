@@ -141,6 +141,34 @@ def test_cta_pair_projection_kernel_equals_single_cta_kernel(kw):
         pu.check_layer_against_oracle(L, wl, b)
 
 
+def test_compress_call_can_be_captured_in_a_cuda_graph_and_replayed():
+    # the whole path (nine launches, tensor maps passed by value) captured once and replayed on new input contents
+    from paper_2502_03805_b200 import session_for, to_device, to_host
+    wl = small_workload(cfg_id=133, dtype="bf16", n=1500, w=32, kp=7, budget_mode="adaptive", budget=600, dh=128,
+                        dm=512, Hq=8, Hkv=2)
+    Ls = [make_layer(wl, l) for l in (0, 1)]
+    bufs = [to_device(getattr(Ls[0], k)[None], "bf16") for k in ("Qw_store", "K_store", "V_store", "WO_store")]
+    s = session_for(wl, nb=1)
+    s.compress(*bufs)                      # first call outside the capture (function attributes, tensor-map entry point)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        s.compress(*bufs, stream=side)
+        graph.capture_end()
+    for L in (Ls[1], Ls[0]):
+        for dst, k in zip(bufs, ("Qw_store", "K_store", "V_store", "WO_store")):
+            dst.copy_(to_device(getattr(L, k)[None], "bf16"))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert s.device_status() == 0
+        out = dict(attn=to_host(s.attn[0]), vnorm=to_host(s.vnorm[0]), idx=to_host(s.idx[0]),
+                   offsets=to_host(s.offsets[0]), stage=to_host(s.stage[0]), K_out=to_host(s.K_out[0]),
+                   V_out=to_host(s.V_out[0]))
+        pu.check_layer_against_oracle(L, wl, out)
+
+
 def test_separate_calls_equal_fused_call_and_are_deterministic():
     wl = small_workload(cfg_id=130, dtype="bf16", n=900, w=32, kp=7, budget=120, dh=128, dm=256)
     _, a, _ = _run(wl)
