@@ -100,6 +100,18 @@ __device__ __forceinline__ void umma_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
+// ---- register reallocation between warpgroups ---------------------------------------------------------------------
+// Every warp of a warpgroup (four consecutive warps) executes the same call.  The kernel is compiled for a fixed
+// register count (launch bounds); role warps that need few registers give theirs back, arithmetic warps take them.
+template <int kRegs>
+__device__ __forceinline__ void warpgroup_reg_dealloc() {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+template <int kRegs>
+__device__ __forceinline__ void warpgroup_reg_alloc() {
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegs));
+}
+
 // ---- CTA pairs (thread-block clusters of two, tcgen05 cta_group::2) --------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;

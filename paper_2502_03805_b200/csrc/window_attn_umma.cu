@@ -17,7 +17,8 @@
 // like the causally invisible ones.
 //
 // Persistent kernel, one CTA per SM: warp 0 streams K tiles (and the group's Q rows, once per work item) with TMA,
-// warp 1 issues the MMAs, warps 2-9 are two sets of four softmax warps that take alternating accumulators (two
+// warp 1 issues the MMAs (warps 2-3 only fill the role warpgroup, which gives its registers to the others with
+// setmaxnreg), warps 4-11 are two sets of four softmax warps that take alternating accumulators (two
 // 256-column TMEM slots), so that the exponentials of one tile overlap the MMAs and TMEM loads of the next.
 // The per-element work is one fma and one exp (plus a max in sweep 1): the normaliser 1 / (w * sum) enters sweep 2
 // as log2 in the exponent's bias, and every reduction runs as four independent chains.
@@ -37,7 +38,11 @@ using namespace ptx;
 constexpr int kKeyTile = 128;
 // softmax warps per (accumulator, TMEM lane quarter); 2 (columns split between two warps) measured no faster
 constexpr int kHalves = 1;
-constexpr int kThreads = (2 + 8 * kHalves) * 32;
+constexpr int kThreads = (4 + 8 * kHalves) * 32;   // warpgroup 0: producer, MMA issuer, two idle warps; then softmax warps
+// launch bounds of 384 threads give every thread 168 registers; the role warpgroup hands most of its share to the
+// softmax warpgroups, whose 128 accumulator values per thread otherwise leave no room to pipeline the exponentials
+constexpr int kRoleRegs = 56, kSoftmaxRegs = 224;
+static_assert(kHalves == 1 && 128 * kRoleRegs + 256 * kSoftmaxRegs <= 65536, "register budget of one CTA per SM");
 constexpr int kSlotCols = 256;
 constexpr int kMaxRowBlocks = 3;  // query rows per work item <= 384
 constexpr float kLog2e = 1.4426950408889634f;
@@ -165,6 +170,8 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 
   bool failed = false;
 
+  if (warp < 4) {
+  warpgroup_reg_dealloc<kRoleRegs>();
   if (warp == 0) {
     // ---------------- producer: Q rows (+ row statistics) per item, K tiles ----------------
     if (lane == 0) {
@@ -272,12 +279,14 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
       umma_commit(drain_bar);
       mbar_wait_bounded(drain_bar, 0, never, 500000000ull);
     }
+  }
   } else {
+    warpgroup_reg_alloc<kSoftmaxRegs>();
     // ---------------- softmax warps ----------------
-    // warp e = warp - 2: TMEM lane quarter = warp % 4 (fixed by the hardware), accumulator slot ("set") = (e / 4) % 2,
+    // warp e = warp - 4: TMEM lane quarter = warp % 4 (fixed by the hardware), accumulator slot ("set") = (e / 4) % 2,
     // column half = e / 8.  A set takes the accumulators with t % 2 == set; its kHalves warps per lane quarter split
     // the columns (sweep 1: keys, sweep 2: heads) between them.
-    const int e_id = warp - 2;
+    const int e_id = warp - 4;
     const uint32_t set = (uint32_t)(e_id >> 2) & 1u;
     const int half = e_id >> 3;
     const int quad = warp & 3;
