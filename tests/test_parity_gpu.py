@@ -418,6 +418,28 @@ def test_right_aligned_ragged_heads_match_the_per_head_oracle(dtype, mode, budge
                                outs[0]["V_out"])
 
 
+@pytest.mark.parametrize("w,dtype", [(128, "bf16"), (256, "bf16"), (100, "f32")])
+def test_ragged_heads_with_long_windows_and_two_slices(w, dtype):
+    # valid_from is per (slice, KV head): two layers with different offsets in one call, windows beyond 64 rows
+    from gen import f32_to_bf16_bits
+    from gpu_util import run_layers
+    wl = small_workload(cfg_id=231, dtype=dtype, n=1700, w=w, kp=5, budget_mode="adaptive", budget=800,
+                        dh=128 if dtype == "bf16" else 64, dm=256, Hq=4, Hkv=2)
+    Ls = [make_layer(wl, l) for l in (0, 1)]
+    cuts = [[0, 333], [640, 1]]
+    fill = f32_to_bf16_bits(np.float32(30.0)) if dtype == "bf16" else np.float32(30.0)
+    for L, cut in zip(Ls, cuts):
+        for g in range(wl.Hkv):
+            L.K_store[g, :cut[g]] = fill
+            L.V_store[g, :cut[g]] = fill
+    vf = torch.tensor(cuts, dtype=torch.int32, device="cuda")
+    outs, s = run_layers(Ls, wl, valid_from=vf)
+    for L, cut, out in zip(Ls, cuts, outs):
+        K_lists = [L.K[g][cut[g]:] for g in range(wl.Hkv)]
+        V_lists = [L.V[g][cut[g]:] for g in range(wl.Hkv)]
+        _check_ragged_call(L.Qw, K_lists, V_lists, L.WO, cut, wl.n, wl, out, "adaptive", wl.budget)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_chunked_prefill_with_adaptive_budgets_matches_oracle_step_by_step(dtype):
     # adaptive budgets leave the heads with different numbers of entries; every step is checked against the oracle run
