@@ -57,7 +57,7 @@ class ShardedCompressor:
     scores of all heads once, and every rank repeats the cheap allocation on the gathered scores."""
 
     def __init__(self, *, nb, Hq, Hkv, dh, dm, n, w, pool_k, dtype, budget_mode, budget, world, rank, alpha=0.5,
-                 eps=1e-4, device=0, gather=all_gather_heads):
+                 eps=1e-4, device=0, gather=all_gather_heads, flags=0, adaptive_floor=0.0, norm=0):
         from . import binding as B
         from .session import CompressionSession
         self.B = B
@@ -65,13 +65,14 @@ class ShardedCompressor:
         G = Hq // Hkv
         hkv_loc = self.g1 - self.g0
         self.global_desc = B.make_desc(nb=nb, Hq=Hq, Hkv=Hkv, dh=dh, dm=dm, n=n, w=w, pool_k=pool_k, dtype=dtype,
-                                       budget_mode=budget_mode, budget=budget, alpha=alpha, eps=eps)
+                                       budget_mode=budget_mode, budget=budget, alpha=alpha, eps=eps, flags=flags,
+                                       adaptive_floor=adaptive_floor, norm=norm)
         self.adaptive = budget_mode == "adaptive"
         local_mode = "given" if self.adaptive else budget_mode
         local_budget = min(budget, hkv_loc * n) if self.adaptive else budget   # capacity of the local outputs
         self.session = CompressionSession(nb=nb, Hq=hkv_loc * G, Hkv=hkv_loc, dh=dh, dm=dm, n=n, w=w, pool_k=pool_k,
                                           dtype=dtype, budget_mode=local_mode, budget=local_budget, alpha=alpha,
-                                          eps=eps, device=device)
+                                          eps=eps, device=device, flags=flags, norm=norm)
         self.gather = gather
         dev = self.session.device
         self.a_local = torch.empty((nb, hkv_loc, n), dtype=torch.float32, device=dev)

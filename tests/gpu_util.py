@@ -14,10 +14,10 @@ def upload_layers(layers, wl, device="cuda:0"):
     return stack("Qw_store"), stack("K_store"), stack("V_store"), stack("WO_store")
 
 
-def run_layers(layers, wl, *, flags=0, separate_calls=False, valid_from=None):
+def run_layers(layers, wl, *, flags=0, separate_calls=False, valid_from=None, **session_kw):
     """One library call over nb = len(layers).  Returns (list of per-layer dicts of host arrays, session)."""
     Qw, K, V, WO = upload_layers(layers, wl)
-    s = session_for(wl, nb=len(layers), flags=flags, valid_from=valid_from)
+    s = session_for(wl, nb=len(layers), flags=flags, valid_from=valid_from, **session_kw)
     if separate_calls:
         s.score(Qw, K, V, WO)
         s.select()

@@ -537,19 +537,23 @@ def test_l2_norm_variant(kw, tensor_cores):
 
 
 @pytest.mark.parametrize("world", [2, 4])
-def test_kv_head_sharded_adaptive_compression_equals_unsharded(world):
+@pytest.mark.parametrize("variant", ["plain", "group_sum_floor"])
+def test_kv_head_sharded_adaptive_compression_equals_unsharded(world, variant):
     # the ranks of a KV-head-sharded layer are played one after the other on this GPU; the all-gather of the group
     # scores is a concatenation.  Every rank must end up with exactly the rows the unsharded call keeps for its heads.
-    from paper_2502_03805_b200 import to_device, to_host
+    from paper_2502_03805_b200 import binding as B, to_device, to_host
     from paper_2502_03805_b200.dist_util import ShardedCompressor
+    flags = B.CKV_FLAG_WO_GROUP_SUM if variant == "group_sum_floor" else 0
+    floor = 0.25 if variant == "group_sum_floor" else 0.0
     wl = small_workload(cfg_id=210, dtype="bf16", n=1800, w=32, kp=7, budget_mode="adaptive", budget=1500, dh=128,
                         dm=512, Hq=16, Hkv=4)
-    Ls, full, _ = _run(wl)
+    Ls, full, _ = _run(wl, flags=flags, adaptive_floor=floor)
     L, ref = Ls[0], full[0]
     shards, a_parts = [], []
     for rank in range(world):
         sc = ShardedCompressor(nb=1, Hq=wl.Hq, Hkv=wl.Hkv, dh=wl.dh, dm=wl.dm, n=wl.n, w=wl.w, pool_k=wl.kp,
-                               dtype="bf16", budget_mode="adaptive", budget=wl.budget, world=world, rank=rank)
+                               dtype="bf16", budget_mode="adaptive", budget=wl.budget, world=world, rank=rank,
+                               flags=flags, adaptive_floor=floor)
         g0, g1 = sc.g0, sc.g1
         h0, h1 = g0 * wl.G, g1 * wl.G
         t = [to_device(np.ascontiguousarray(x)[None], "bf16")
