@@ -241,8 +241,12 @@ def main():
     t0 = time.time()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record(stream)
+    step_ev = [ev0]
     for _ in range(args.steps):
         step(record=True)
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        step_ev.append(e)
     ev1.record(stream)
     barrier()
     t1 = time.time()
@@ -251,6 +255,7 @@ def main():
     assert s.device_status() == 0, "device status word set during the timed region"
     ms_total = ev0.elapsed_time(ev1)
     gemm_ms = [a.elapsed_time(b) for a, b in gemm_ev]
+    per_step = sorted(a.elapsed_time(b) for a, b in zip(step_ev[:-1], step_ev[1:]))
     path = s.last_path
 
     # ---- per-stage device times, taken after the timed region (three more steps with events between the stages) ----
@@ -340,7 +345,8 @@ def main():
             cpu = {"value": entries / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
                    "sample": f"layer 0 of {wl.layers} (all heads, full n={wl.n}), {dt:.1f} s; numpy float64"}
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "ms_per_step_median": per_step[len(per_step) // 2],
+                "ms_per_step_min": per_step[0], "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "bf16" if wl.dtype == "bf16" else "f32", "data": "synthetic",
                 "config": {"workload": wl.name, "layers": nb, "Hq": wl.Hq, "Hkv": wl.Hkv, "head_dim": wl.dh,
                            "d_model": wl.dm, "n": wl.n, "window": wl.w, "pool_kernel": wl.kp,
