@@ -14,7 +14,9 @@ struct criticalkv_handle_s {
   int sm_count;
   int cc_major, cc_minor;
   int* status_word;  // device
+  int smem_optin;
   int last_path;
+  int last_select_fused;
   long long launches;
   char cuda_error[256];
   // host-staged path: two copy/compute streams and the events that tie them to the caller's stream
@@ -55,7 +57,8 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (d->reserved != 0 || d->reserved2 != 0) return CKV_EINVAL;
   if (!(d->adaptive_floor >= 0.f && d->adaptive_floor <= 1.f)) return CKV_EINVAL;
   if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM |
-                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_CTA_PAIR_MMA)) return CKV_EINVAL;
+                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_CTA_PAIR_MMA | CKV_FLAG_SELECT_MULTIPASS))
+    return CKV_EINVAL;
   if (d->budget < 0) return CKV_EINVAL;
   if ((long long)d->n * d->Hkv > 0x7fffffffLL) return CKV_ENOTSUP;
   o->nb = d->nb; o->Hq = d->Hq; o->Hkv = d->Hkv; o->G = d->Hq / d->Hkv;
@@ -176,6 +179,7 @@ int criticalkv_create(criticalkv_handle* out, int device) {
   h->sm_count = prop.multiProcessorCount;
   h->cc_major = prop.major;
   h->cc_minor = prop.minor;
+  h->smem_optin = (int)prop.sharedMemPerBlockOptin;
   *out = h;
   return CKV_OK;
 }
@@ -299,8 +303,9 @@ int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, const float
   char* base = (char*)ws;
   ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets)};
   int launches = 0;
-  cudaError_t e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, (cudaStream_t)stream,
-                                     &launches, h->status_word);
+  const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1};
+  cudaError_t e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, sd, (cudaStream_t)stream,
+                                     &launches, h->status_word, &h->last_select_fused);
   h->launches += launches;
   return record_cuda(h, e);
 }
@@ -644,8 +649,9 @@ int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc* d, cons
   char* base = (char*)scratch;
   ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets)};
   int launches = 0;
-  e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, (cudaStream_t)stream, &launches,
-                         h->status_word);
+  const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1};
+  e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, sd, (cudaStream_t)stream, &launches,
+                         h->status_word, &h->last_select_fused);
   h->launches += launches;
   return record_cuda(h, e);
 }
@@ -664,7 +670,7 @@ const char* criticalkv_status_string(int s) {
 }
 
 const char* criticalkv_last_cuda_error(criticalkv_handle h) { return h ? h->cuda_error : ""; }
-int criticalkv_last_path(criticalkv_handle h) { return h ? h->last_path : 0; }
+int criticalkv_last_path(criticalkv_handle h) { return h ? (h->last_path | (h->last_select_fused ? 32 : 0)) : 0; }
 int64_t criticalkv_launch_count(criticalkv_handle h) { return h ? h->launches : 0; }
 
 }  // extern "C"

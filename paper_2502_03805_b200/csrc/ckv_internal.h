@@ -83,9 +83,21 @@ cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* v
                                 cudaStream_t st, int* launches);
 cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* budgets_out, cudaStream_t st,
                                     int* launches);
+// What the selection launcher needs to know about the device and the caller's wishes.
+struct SelectDevice {
+  int sm_count;
+  int smem_optin;    // largest dynamic shared memory a CTA may ask for
+  int allow_fused;   // 0: always the multi-kernel path (CKV_FLAG_SELECT_MULTIPASS)
+};
+// *fused = 1 when the single-kernel path ran.
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
-                          cudaStream_t st, int* launches, int* status_word);
+                          const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word, int* fused);
+// Steps 3-4 as one kernel (keys of a head in shared memory).  cudaErrorNotSupported = the shape does not fit or the
+// cluster launch is not available; nothing has been launched then.
+cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
+                                int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
+                                int smem_limit, cudaStream_t st, int* launches, int* status_word);
 cudaError_t launch_compact(const Dims& d, const void* K, const void* V, const int32_t* idx, const int32_t* offsets,
                            void* K_out, void* V_out, cudaStream_t st, int* launches);
 
