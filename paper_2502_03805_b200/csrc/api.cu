@@ -129,15 +129,19 @@ ScoreLayout score_layout(const Dims& d) {
   return L;
 }
 struct SelectLayout {
-  size_t a, c, budgets, total;
+  size_t a, c, budgets, sync, sync_bytes, total;
 };
-SelectLayout select_layout(const Dims& d) {
+// with_sync: room for the per-slice block the single-kernel selection needs for adaptive budgets
+SelectLayout select_layout(const Dims& d, bool with_sync = true) {
   SelectLayout L;
-  const size_t per = (size_t)d.nb * d.Hkv * d.n * sizeof(float);
+  const size_t per = (size_t)d.nb * d.Hkv * ckv::select_head_stride(d.n) * sizeof(float);
   size_t off = 0;
   L.a = off; off = align_up(off + per, 256);
   L.c = off; off = align_up(off + per, 256);
   L.budgets = off; off = align_up(off + (size_t)d.nb * d.Hkv * sizeof(int32_t), 256);
+  L.sync = off;
+  L.sync_bytes = with_sync ? ckv::select_sync_bytes(d) : 0;
+  off = align_up(off + L.sync_bytes, 256);
   L.total = off;
   return L;
 }
@@ -301,7 +305,8 @@ int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, const float
   DeviceGuard guard(h->device);
   if (!guard.ok) return CKV_ECUDA;
   char* base = (char*)ws;
-  ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets)};
+  ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets),
+                          L.sync_bytes ? (void*)(base + L.sync) : nullptr};
   int launches = 0;
   const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1};
   cudaError_t e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, sd, (cudaStream_t)stream,
@@ -634,7 +639,7 @@ int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc* d, cons
   if (!aligned16(attn) || !aligned16(vnorm) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
       (reinterpret_cast<uintptr_t>(offsets) & 3u) || (reinterpret_cast<uintptr_t>(budgets_in) & 3u))
     return CKV_EALIGN;
-  const SelectLayout L = select_layout(dd);
+  const SelectLayout L = select_layout(dd, false);
   if (L.total > CKV_STATIC_SCRATCH_BYTES) {
     snprintf(h->cuda_error, sizeof(h->cuda_error),
              "criticalkv_select_static: this shape needs %zu bytes of scratch, the built-in array holds %zu",
@@ -647,7 +652,8 @@ int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc* d, cons
   cudaError_t e = static_scratch_address(h->device, &scratch);
   if (e != cudaSuccess) return record_cuda(h, e);
   char* base = (char*)scratch;
-  ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets)};
+  ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets),
+                          L.sync_bytes ? (void*)(base + L.sync) : nullptr};
   int launches = 0;
   const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1};
   e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, sd, (cudaStream_t)stream, &launches,

@@ -37,10 +37,14 @@ struct ScoreWorkspace {   // carved out of the caller's workspace by the API lay
 };
 
 struct SelectWorkspace {
-  float* a;         // [nb, Hkv, n]
-  float* c;         // [nb, Hkv, n]
+  float* a;         // [nb, Hkv, n]  (single-kernel path: integer keys, [nb*Hkv][32][words], see select_fused.cu)
+  float* c;         // [nb, Hkv, n]  (same)
   int32_t* budgets; // [nb, Hkv]
+  void* sync;       // select_sync_bytes(): per-slice histograms and barrier counters of the single-kernel path, or null
 };
+// Floats per head in each of the regions a and c: n rounded up to a whole, even number of 32-entry words.
+inline size_t select_head_stride(int n) { return (size_t)32 * ((((size_t)n + 31) / 32 + 1) & ~(size_t)1); }
+size_t select_sync_bytes(const Dims& d);
 
 // ---- launchers (each returns the first CUDA error of its launches) ----
 cudaError_t launch_window_attn_simt(const Dims& d, const void* Qw, const void* K, float* attn,
@@ -93,11 +97,11 @@ struct SelectDevice {
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word, int* fused);
-// Steps 3-4 as one kernel (keys of a head in shared memory).  cudaErrorNotSupported = the shape does not fit or the
-// cluster launch is not available; nothing has been launched then.
+// Steps 3-4 as one kernel.  cudaErrorNotSupported = the shape is outside what it handles or the cooperative launch is
+// not available; no kernel has been launched then.
 cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                                 int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
-                                int smem_limit, cudaStream_t st, int* launches, int* status_word);
+                                const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word);
 cudaError_t launch_compact(const Dims& d, const void* K, const void* V, const int32_t* idx, const int32_t* offsets,
                            void* K_out, void* V_out, cudaStream_t st, int* launches);
 

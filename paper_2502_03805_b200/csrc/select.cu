@@ -335,9 +335,9 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
                           const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word, int* fused) {
   *fused = 0;
   if (dev.allow_fused) {
-    // one kernel when a head's keys fit in shared memory; otherwise the three kernels below
-    const cudaError_t ef = launch_select_fused(d, attn, vnorm, budgets_in, idx, offsets, stage, ws, dev.smem_optin,
-                                               st, launches, status_word);
+    // one kernel when the shape allows it; otherwise the three kernels below
+    const cudaError_t ef = launch_select_fused(d, attn, vnorm, budgets_in, idx, offsets, stage, ws, dev, st, launches,
+                                               status_word);
     if (ef == cudaSuccess) {
       *fused = 1;
       return ef;

@@ -1,67 +1,116 @@
-// Steps 3-4 in ONE kernel for heads whose attention keys fit in shared memory (Algorithm 1: scores, b' = floor(alpha b),
-// stage 1 by attention, stage 2 by the perturbation-aware score among the rest; Algorithm 2: budget allocation).
+// Steps 3-4 in ONE kernel (Algorithm 1: scores, b' = floor(alpha b), stage 1 by attention, stage 2 by the
+// perturbation-aware score among the rest; Algorithm 2: budget allocation across the heads of a layer).
 //
-// One CTA per (nb slice, KV head).  attn and vnorm are read from memory exactly once:
+// A CTA works on one (nb slice, KV head) at a time; attn and vnorm cross HBM exactly once:
 //   reduce   : a_g, c_g from the group's query heads in the fixed float32 operation order of the selection (see
-//              select.cu); the order-preserving integer keys of a_g stay in shared memory, c_g goes to a scratch
-//              array that this CTA alone re-reads (twice, from L2); the 12-bit first-digit histogram of a_g is built
+//              select.cu), turned into order-preserving integer keys and written to a scratch array in a
+//              word-transposed layout (entry i = 32 t + j lives at [j][t]), so that later walks give every thread
+//              whole 32-entry words with coalesced loads; the 12-bit first-digit histograms of a_g and c_g are built
 //              on the way
-//   budgets  : flattened adaptive allocation across the KV heads of a slice = the CTAs of one thread-block cluster:
-//              three radix rounds (12 + 10 + 10 bits), histograms summed through distributed shared memory
-//   stage 1  : radix select on the shared-memory keys (first round = the histogram already built), ordered marking
-//              walk (ties to the lower index) that at the same time builds the first-digit histogram of c over the
-//              entries stage 1 left
-//   stage 2  : one walk over c marks the entries above the threshold bin and collects the entries inside it; the
-//              remaining digits and the index tie-break run on that short list
-//   output   : ordered compaction of the two bit masks into ascending indices
-// Every decision is taken on the same integer keys and with the same tie rule as the multi-kernel path, so both give
-// identical results.  Shapes that do not fit (keys beyond shared memory, more KV heads than a portable cluster) are
-// left to the multi-kernel path.
-#include <cooperative_groups.h>
-
+//   budgets  : flattened adaptive allocation over the KV heads of a slice, i.e. over several CTAs: the first-digit
+//              histograms are summed in a per-slice block of global memory, every CTA publishes its keys of the
+//              threshold bin, and each CTA then finishes the selection on the union of those short lists; two
+//              bounded barriers per slice (the launch is cooperative, so all CTAs are resident).  Lists that do not
+//              fit fall back to two more histogram rounds with a barrier each
+//   stage 1  : one walk over a and c marks the entries above the threshold bin, collects the entries inside it
+//              (remaining digits and index tie-break run on that short list) and counts the first digit of c for
+//              the entries stage 1 leaves, restricted to the bins the stage-2 threshold can fall into
+//   stage 2  : one walk over c marks the entries above the threshold bin and collects the entries inside it
+//   output   : ordered compaction of the two bit masks into ascending indices, written in coalesced runs
+// The scratch arrays are re-read from L2 (a once or twice, c twice); two CTAs share an SM.  Every decision is taken on
+// the same integer keys and with the same tie rule as the multi-kernel path: both give identical results.  Scores
+// must not be NaN (the padding of the last word uses the key 0, which only a NaN bit pattern maps to).
 #include "ckv_internal.h"
 #include "select_common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace ckv {
 namespace {
 
-namespace cg = cooperative_groups;
-
+constexpr int kFT = 512;                       // threads per CTA
+constexpr int kFW = kFT / 32;
 constexpr int kD1Shift = 20, kD1Bins = 4096;   // first digit: sign, exponent and 3 mantissa bits
 constexpr int kD2Bins = 1024;                  // second and third digit: 10 bits each
-constexpr int kMaxCluster = 8;                 // portable cluster size
+constexpr int kCandCap = 2048;                 // keys of a threshold bin kept in shared memory
+constexpr int kMaxWords = kD1Bins;             // 32-entry words per head (n <= 131072)
+constexpr int kMaxHeads = 64;
+
+// Per nb slice, zeroed before the launch (adaptive budgets only); followed by Hkv lists of kCandCap keys.
+struct LayerSync {
+  uint32_t hist1[kD1Bins];
+  uint32_t hist2[kD2Bins];
+  uint32_t hist3[kD2Bins];
+  uint32_t cnt[kMaxHeads][2];   // fallback rounds: keys above / equal to the flattened threshold per KV head
+  uint32_t ncand[kMaxHeads];    // keys of the threshold bin per KV head
+  uint32_t above[kMaxHeads];    // keys in higher bins per KV head
+  uint32_t arrive[8];           // one counter per barrier
+  uint32_t overflow;            // some head's list did not fit
+  uint32_t pad[23];
+};
+static_assert(sizeof(LayerSync) % 16 == 0, "slices of the sync block stay 16-byte aligned");
+__host__ __device__ inline size_t layer_sync_stride(int Hkv) {
+  return sizeof(LayerSync) + (size_t)Hkv * kCandCap * sizeof(uint32_t);
+}
 
 struct FusedArgs {
   const float* attn;
   const float* vnorm;
   const int32_t* budgets_in;   // given budgets [nb, Hkv] or null
-  float* c;                    // scratch [nb, Hkv, n]
-  int32_t* budgets_out;        // [nb, Hkv]: the budgets actually used (adaptive mode), may be null
+  uint32_t* a_t;               // scratch: keys of a, [nb*Hkv][32][nw]
+  uint32_t* c_t;               // scratch: keys of c, same layout
+  uint8_t* sync;               // [nb] blocks of layer_sync_stride(Hkv) bytes (adaptive only)
+  int32_t* budgets_out;        // [nb, Hkv]: the budgets used (adaptive mode), may be null
   int32_t* idx;
   int32_t* offsets;
   uint8_t* stage;
   int* status;
   const int32_t* valid_from;
-  int Hq, Hkv, G, n;
+  int Hq, Hkv, G, n, nw;       // nw: words per head, even
   int group_sum, protect_from;
-  int cand_cap;
+  long long nitems;
   long long uniform_b, btot, b_adapt;
   int floor_b;
   float alpha, eps;
 };
 
-struct FusedFixed {
-  SelectShared old;          // hist[0..15] = first-digit histogram of a, hist[16..31] = working histogram
-  uint32_t wtot[kSelWarps];
-  uint32_t res_bin, res_k;
-  uint32_t cand_count;
-  uint32_t cnt[2];           // this head's keys above / equal to the flattened threshold (read by the cluster)
+struct FusedShared {
+  uint32_t hist_a[kD1Bins];    // first-digit histogram of a; afterwards scratch (list rounds, tie prefixes)
+  uint32_t hist_c[kD1Bins];    // first-digit histogram of c over all entries
+  uint32_t hist_w[kD1Bins];    // working histogram
+  uint32_t cand_key[kCandCap];
+  uint32_t cand_idx[kCandCap];
+  uint32_t cand_c[kCandCap];
+  uint32_t head_cnt[kMaxHeads][2];
+  uint32_t wtot[kFW];
+  uint32_t res_bin, res_k, cand_count, flag;
+  uint32_t red[4];
 };
 
-// k-th largest position in a histogram spread over the CTA: thread t holds the counts of bins t*PER .. t*PER+PER-1
-// (higher bin = larger key).  Returns the bin that holds the k-th largest key and k minus the keys in higher bins.
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t lanemask_lt() {
+  uint32_t m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+// Slot in a list for every calling thread; the threads of a warp that call together share one atomic.
+__device__ __forceinline__ uint32_t list_slot(uint32_t* counter) {
+  const uint32_t m = __activemask();
+  const int leader = __ffs(m) - 1;
+  uint32_t base = 0;
+  if ((int)(threadIdx.x & 31) == leader) base = atomicAdd(counter, (uint32_t)__popc(m));
+  base = __shfl_sync(m, base, leader);
+  return base + __popc(m & lanemask_lt());
+}
+
+// Bin of the k-th largest key in a histogram spread over the CTA: thread t holds bins t*PER .. t*PER+PER-1 (higher
+// bin = larger key).  Returns the bin and k minus the keys in higher bins (all threads).
 template <int PER>
-__device__ __forceinline__ void find_bin(const uint32_t (&v)[PER], uint32_t k, FusedFixed& sh, uint32_t* bin,
+__device__ __forceinline__ void find_bin(const uint32_t (&v)[PER], uint32_t k, FusedShared& sh, uint32_t* bin,
                                          uint32_t* krem) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   uint32_t s = 0;
@@ -74,10 +123,15 @@ __device__ __forceinline__ void find_bin(const uint32_t (&v)[PER], uint32_t k, F
     if (lane + o < 32) x += y;
   }
   if (lane == 0) sh.wtot[warp] = x;
-  if (tid == 0) { sh.res_bin = 0; sh.res_k = 0; }
   __syncthreads();
+  // the result words are written only between the two barriers: a thread that is still reading the previous call's
+  // result has not reached the first one yet
   uint32_t above = x - s;
-  for (int q = warp + 1; q < kSelWarps; ++q) above += sh.wtot[q];
+  for (int q = warp + 1; q < kFW; ++q) above += sh.wtot[q];
+  if (tid == 0 && (k == 0 || k > above + s)) {   // thread 0 sees the total: k outside the histogram
+    sh.res_bin = 0;
+    sh.res_k = 0;
+  }
   if (s > 0 && above < k && k <= above + s) {
     uint32_t acc = above;
 #pragma unroll
@@ -94,443 +148,802 @@ __device__ __forceinline__ void find_bin(const uint32_t (&v)[PER], uint32_t k, F
   *bin = sh.res_bin;
   *krem = sh.res_k;
 }
+// The same over a histogram in shared memory.
+__device__ __forceinline__ void find_bin_d1(const uint32_t* hist, uint32_t k, FusedShared& sh, uint32_t* bin,
+                                            uint32_t* krem) {
+  uint32_t v[8];
+  const uint4 x = *reinterpret_cast<const uint4*>(hist + 8 * threadIdx.x);
+  const uint4 y = *reinterpret_cast<const uint4*>(hist + 8 * threadIdx.x + 4);
+  v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
+  find_bin<8>(v, k, sh, bin, krem);
+}
+__device__ __forceinline__ void find_bin_d2(const uint32_t* hist, uint32_t k, FusedShared& sh, uint32_t* bin,
+                                            uint32_t* krem) {
+  uint32_t v[2] = {hist[2 * threadIdx.x], hist[2 * threadIdx.x + 1]};
+  find_bin<2>(v, k, sh, bin, krem);
+}
+
+// Exclusive prefix of v over the threads of the CTA (thread order) and the CTA-wide total.
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, FusedShared& sh, uint32_t* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  uint32_t x = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t y = __shfl_up_sync(0xffffffffu, x, o);
+    if (lane >= o) x += y;
+  }
+  if (lane == 31) sh.wtot[warp] = x;
+  __syncthreads();
+  uint32_t before = 0, all = 0;
+  for (int q = 0; q < kFW; ++q) {
+    const uint32_t w = sh.wtot[q];
+    if (q < warp) before += w;
+    all += w;
+  }
+  __syncthreads();
+  *total = all;
+  return before + x - v;
+}
+__device__ __forceinline__ uint32_t block_sum(uint32_t v, FusedShared& sh) {
+  uint32_t total;
+  (void)block_excl_scan(v, sh, &total);
+  return total;
+}
 
 __device__ __forceinline__ void zero_words(uint32_t* p, int count) {
-  for (int e = threadIdx.x; e < count; e += kSelThreads) p[e] = 0;
+  for (int e = threadIdx.x; e < count; e += kFT) p[e] = 0;
+}
+
+// The CTAs that work on the heads of one slice meet here.  Bounded: gives up after two seconds (false).
+__device__ __forceinline__ bool layer_barrier(uint32_t* counter, uint32_t target, FusedShared& sh) {
+  __syncthreads();   // every thread's writes and reductions to the slice's block are issued
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(counter, 1u);
+    bool ok = true;
+    if (ld_acquire(counter) < target) {
+      const uint64_t t0 = ptx::global_timer_ns();
+      for (uint32_t spin = 1;; ++spin) {
+        if (ld_acquire(counter) >= target) break;
+        if ((spin & 63u) == 0 && ptx::global_timer_ns() - t0 > 2000000000ull) {
+          ok = false;
+          break;
+        }
+      }
+    }
+    __threadfence();
+    sh.flag = ok ? 1u : 0u;
+  }
+  __syncthreads();
+  return sh.flag != 0;
 }
 
 // One entry of the group reduce: the sums over the group's heads are finished into (a, c), the special scores of the
 // protected window and of the padding are applied, and -0 is folded into +0.
-__device__ __forceinline__ void finish_entry(float sa, float sc, float Gf, float eps, int group_sum, float vg, int i,
-                                             int protect_from, int vf, float* av_out, float* cv_out) {
-  float av = __fdiv_rn(sa, Gf);
-  float cv = group_sum ? __fmul_rn(__fadd_rn(av, eps), vg) : __fdiv_rn(sc, Gf);
+__device__ __forceinline__ void finish_entry(float sa, float sc, float Gf, float invG, bool pow2, float eps,
+                                             int group_sum, float vg, int i, int protect_from, int vf,
+                                             uint32_t* ka, uint32_t* kc) {
+  // dividing by a power of two and multiplying by its reciprocal round the same exact value
+  float av = pow2 ? __fmul_rn(sa, invG) : __fdiv_rn(sa, Gf);
+  float cv = group_sum ? __fmul_rn(__fadd_rn(av, eps), vg) : (pow2 ? __fmul_rn(sc, invG) : __fdiv_rn(sc, Gf));
   if (i >= protect_from) av = cv = 3.402823466e+38f;
   if (i < vf) av = cv = -1.0f;
   if (av == 0.f) av = 0.f;
   if (cv == 0.f) cv = 0.f;
-  *av_out = av;
-  *cv_out = cv;
+  *ka = order_key(av);
+  *kc = order_key(cv);
 }
 
-template <bool kCluster>
-__global__ void __launch_bounds__(kSelThreads, 1) select_fused_kernel(FusedArgs p) {
-  extern __shared__ __align__(16) uint8_t fused_smem[];
-  FusedFixed& sh = *reinterpret_cast<FusedFixed*>(fused_smem);
-  const int n = p.n;
-  const int nwords = (n + 31) / 32;
-  uint32_t* keys = reinterpret_cast<uint32_t*>(fused_smem + ((sizeof(FusedFixed) + 15) / 16) * 16);
-  uint32_t* sel1 = keys + ((n + 3) / 4) * 4;
-  uint32_t* sel2 = sel1 + nwords;
-  uint32_t* cand_key = sel2 + nwords;
-  uint32_t* cand_idx = cand_key + p.cand_cap;
-  uint32_t* hist_d1 = &sh.old.hist[0][0];
-  uint32_t* hist_w = &sh.old.hist[kSelWarps / 2][0];
-  static_assert(kSelWarps * 256 == 2 * kD1Bins, "the two histograms alias the 8-bit select's per-warp histograms");
-
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int b = blockIdx.x / p.Hkv, g = blockIdx.x % p.Hkv;
-  const int G = p.G;
-  const long long h0 = (long long)b * p.Hq + (long long)g * G;
-  const float Gf = (float)G;
-  const int vf = p.valid_from ? p.valid_from[b * p.Hkv + g] : 0;
-  float* cg_out = p.c + ((long long)b * p.Hkv + g) * n;
-
-  zero_words(hist_d1, 2 * kD1Bins);
-  if (tid == 0) { sh.cand_count = 0; sh.cnt[0] = 0; sh.cnt[1] = 0; }
-  __syncthreads();
-
-  // ---------------- reduce: one pass over attn and vnorm ----------------
-  const float* vg_row = p.group_sum ? p.vnorm + ((long long)b * p.Hkv + g) * n : nullptr;
-  if ((n & 3) == 0) {
-    const int n4 = n >> 2;
-    for (int i4 = tid; i4 < n4; i4 += kSelThreads) {
-      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sc[4] = {0.f, 0.f, 0.f, 0.f};
-      for (int q0 = 0; q0 < G; q0 += 4) {
-        float4 pa[4], pv[4];
+// Four consecutive keys into a first-digit histogram: neighbours mostly share a bin, one atomic per run.
+__device__ __forceinline__ void count_digits4(uint32_t* hist, const uint32_t (&k)[4]) {
+  uint32_t cur = k[0] >> kD1Shift, run = 1;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (q0 + u < G) {
-            pa[u] = __ldcs(reinterpret_cast<const float4*>(p.attn + (h0 + q0 + u) * n) + i4);
-            if (!p.group_sum) pv[u] = __ldcs(reinterpret_cast<const float4*>(p.vnorm + (h0 + q0 + u) * n) + i4);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (q0 + u < G) {
-            const float a4[4] = {pa[u].x, pa[u].y, pa[u].z, pa[u].w};
-            float v4[4] = {0.f, 0.f, 0.f, 0.f};
-            if (!p.group_sum) { v4[0] = pv[u].x; v4[1] = pv[u].y; v4[2] = pv[u].z; v4[3] = pv[u].w; }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float prod = __fmul_rn(__fadd_rn(a4[j], p.eps), v4[j]);
-              if (q0 + u == 0) { sa[j] = a4[j]; sc[j] = prod; }
-              else { sa[j] = __fadd_rn(sa[j], a4[j]); sc[j] = __fadd_rn(sc[j], prod); }
-            }
-          }
-        }
-      }
-      float4 vg4 = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (p.group_sum) vg4 = __ldcs(reinterpret_cast<const float4*>(vg_row) + i4);
-      const float vgs[4] = {vg4.x, vg4.y, vg4.z, vg4.w};
-      float cv[4];
-      uint32_t ka[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        float av;
-        finish_entry(sa[j], sc[j], Gf, p.eps, p.group_sum, vgs[j], 4 * i4 + j, p.protect_from, vf, &av, &cv[j]);
-        ka[j] = order_key(av);
-      }
-      *reinterpret_cast<uint4*>(keys + 4 * i4) = make_uint4(ka[0], ka[1], ka[2], ka[3]);
-      *reinterpret_cast<float4*>(cg_out + 4 * i4) = make_float4(cv[0], cv[1], cv[2], cv[3]);
-      // neighbouring entries mostly share a bin (the scores are max-pooled): one atomic per run
-      uint32_t cur = ka[0] >> kD1Shift, run = 1;
-#pragma unroll
-      for (int j = 1; j < 4; ++j) {
-        const uint32_t bin = ka[j] >> kD1Shift;
-        if (bin == cur) {
-          ++run;
-        } else {
-          atomicAdd(&hist_d1[cur], run);
-          cur = bin;
-          run = 1;
-        }
-      }
-      atomicAdd(&hist_d1[cur], run);
-    }
-  } else {
-    for (int i = tid; i < n; i += kSelThreads) {
-      float sa = 0.f, sc = 0.f;
-      for (int q = 0; q < G; ++q) {
-        const float a1 = p.attn[(h0 + q) * n + i];
-        const float v1 = p.group_sum ? 0.f : p.vnorm[(h0 + q) * n + i];
-        const float prod = __fmul_rn(__fadd_rn(a1, p.eps), v1);
-        if (q == 0) { sa = a1; sc = prod; }
-        else { sa = __fadd_rn(sa, a1); sc = __fadd_rn(sc, prod); }
-      }
-      float av, cv;
-      finish_entry(sa, sc, Gf, p.eps, p.group_sum, p.group_sum ? vg_row[i] : 0.f, i, p.protect_from, vf, &av, &cv);
-      const uint32_t ka = order_key(av);
-      keys[i] = ka;
-      cg_out[i] = cv;
-      atomicAdd(&hist_d1[ka >> kD1Shift], 1u);
-    }
-  }
-  __syncthreads();
-
-  // ---------------- this head's budget and the start of its segment ----------------
-  long long off = 0, bud = 0;
-  bool clipped = false;
-  if (kCluster) {
-    // flattened top-b_adapt over the keys of every head of the slice (the CTAs of this cluster)
-    cg::cluster_group cluster = cg::this_cluster();
-    const int cs = (int)cluster.num_blocks();
-    uint32_t T = 0, r = 0;
-    if (p.b_adapt > 0) {
-      cluster.sync();   // every head's first-digit histogram is complete
-      uint32_t v4[4] = {0u, 0u, 0u, 0u};
-      for (int q = 0; q < cs; ++q) {
-        const uint4 x = *reinterpret_cast<const uint4*>(cluster.map_shared_rank(hist_d1, q) + 4 * tid);
-        v4[0] += x.x; v4[1] += x.y; v4[2] += x.z; v4[3] += x.w;
-      }
-      uint32_t bin, krem;
-      find_bin<4>(v4, (uint32_t)p.b_adapt, sh, &bin, &krem);
-      uint32_t prefix = bin;   // the key bits fixed so far, right-aligned
-      for (int round = 0; round < 2; ++round) {
-        const int shift = round == 0 ? 10 : 0;
-        zero_words(hist_w, kD2Bins);
-        __syncthreads();
-        for (int i = tid; i < n; i += kSelThreads) {
-          const uint32_t key = keys[i];
-          if ((key >> (shift + 10)) == prefix) atomicAdd(&hist_w[(key >> shift) & (kD2Bins - 1)], 1u);
-        }
-        cluster.sync();   // every rank's working histogram is complete
-        uint32_t v1[1] = {0u};
-        for (int q = 0; q < cs; ++q) v1[0] += cluster.map_shared_rank(hist_w, q)[tid];
-        cluster.sync();   // ... and has been read by everyone before the next round clears it
-        find_bin<1>(v1, krem, sh, &bin, &krem);
-        prefix = (prefix << 10) | bin;
-      }
-      T = prefix;
-      r = krem;
-      uint32_t gt = 0, eq = 0;
-      for (int i = tid; i < n; i += kSelThreads) {
-        const uint32_t key = keys[i];
-        gt += key > T;
-        eq += key == T;
-      }
-      gt = __reduce_add_sync(0xffffffffu, gt);
-      eq = __reduce_add_sync(0xffffffffu, eq);
-      if (lane == 0) {
-        if (gt) atomicAdd(&sh.cnt[0], gt);
-        if (eq) atomicAdd(&sh.cnt[1], eq);
-      }
-      cluster.sync();   // every head's counts are complete
-      uint32_t rem = r;
-      for (int q = 0; q < cs; ++q) {
-        const uint32_t* pc = cluster.map_shared_rank(sh.cnt, q);
-        const uint32_t take = min(pc[1], rem);
-        const long long bq = min((long long)pc[0] + take + p.floor_b, (long long)n);
-        rem -= take;
-        if (q < g) off += bq;
-        if (q == g) bud = bq;
-      }
-      cluster.sync();   // nobody leaves (or rewrites cnt) while a peer still reads its shared memory
+  for (int j = 1; j < 4; ++j) {
+    const uint32_t bin = k[j] >> kD1Shift;
+    if (bin == cur) {
+      ++run;
     } else {
-      bud = min((long long)p.floor_b, (long long)n);
-      off = (long long)g * bud;
+      atomicAdd(&hist[cur], run);
+      cur = bin;
+      run = 1;
     }
-    if (off > p.btot) { off = p.btot; clipped = true; }
-    if (off + bud > p.btot) { bud = p.btot - off; clipped = true; }
-    if (p.budgets_out != nullptr && tid == 0) p.budgets_out[(long long)b * p.Hkv + g] = (int32_t)bud;
-  } else if (p.budgets_in == nullptr) {
-    bud = p.uniform_b;
-    off = (long long)g * bud;
-  } else {
-    const int32_t* bb = p.budgets_in + (long long)b * p.Hkv;
-    for (int q = 0; q < g; ++q) off += min(max((long long)bb[q], 0LL), (long long)n);
-    bud = bb[g];
-    if (bud < 0 || bud > n) { bud = min(max(bud, 0LL), (long long)n); clipped = true; }
-    if (off > p.btot) { off = p.btot; clipped = true; }
-    if (off + bud > p.btot) { bud = p.btot - off; clipped = true; }
   }
-  if (clipped && tid == 0) atomicExch(p.status, (int)CKV_EINVAL);
-  long long b1 = (long long)floor((double)p.alpha * (double)bud);
-  b1 = min(max(b1, 0LL), bud);
-  const long long b2 = bud - b1;
+  atomicAdd(&hist[cur], run);
+}
 
-  // ---------------- stage 1: the b1 largest a (keys in shared memory) ----------------
-  uint32_t T1 = 0, r1 = 0;
-  if (b1 > 0) {
-    uint32_t v4[4];
-    {
-      const uint4 x = *reinterpret_cast<const uint4*>(hist_d1 + 4 * tid);
-      v4[0] = x.x; v4[1] = x.y; v4[2] = x.z; v4[3] = x.w;
+// Applies f(key0, key1, j) to the entries j = 0..31 of the word pair (2 wp, 2 wp + 1); eight loads in flight.
+template <typename F>
+__device__ __forceinline__ void walk_pair(const uint32_t* __restrict__ arr, int nw, int wp, F&& f) {
+  const uint2* p = reinterpret_cast<const uint2*>(arr) + wp;
+  const size_t row = (size_t)(nw >> 1);
+#pragma unroll 1
+  for (int j0 = 0; j0 < 32; j0 += 8) {
+    uint2 k[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) k[u] = __ldcg(p + (size_t)(j0 + u) * row);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) f(k[u].x, k[u].y, j0 + u);
+  }
+}
+template <typename F>
+__device__ __forceinline__ void walk_pair2(const uint32_t* __restrict__ arr_a, const uint32_t* __restrict__ arr_b,
+                                           int nw, int wp, F&& f) {
+  const uint2* pa = reinterpret_cast<const uint2*>(arr_a) + wp;
+  const uint2* pb = reinterpret_cast<const uint2*>(arr_b) + wp;
+  const size_t row = (size_t)(nw >> 1);
+#pragma unroll 1
+  for (int j0 = 0; j0 < 32; j0 += 4) {
+    uint2 ka[4], kb[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      ka[u] = __ldcg(pa + (size_t)(j0 + u) * row);
+      kb[u] = __ldcg(pb + (size_t)(j0 + u) * row);
     }
-    uint32_t bin, krem;
-    find_bin<4>(v4, (uint32_t)b1, sh, &bin, &krem);
-    uint32_t prefix = bin;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) f(ka[u].x, ka[u].y, kb[u].x, kb[u].y, j0 + u);
+  }
+}
+
+// Second and third radix round over the keys of `arr` (entries excluded by `excl` skipped) whose first digit is bin1;
+// the first round's result (bin1, krem) comes from a histogram the caller already has.  With kSync the histograms of
+// the rounds are summed over the CTAs of the slice (barriers arrive[2], arrive[3]).  Returns the threshold key T, how
+// many of the keys equal to T belong to the top k (r), how many keys equal T in this CTA's array (own_eq), and adds
+// this CTA's keys in higher bins of rounds two and three to *own_gt.  Uses cand_key as list.  false = a barrier
+// timed out.
+template <bool kExcl, bool kSync>
+__device__ __forceinline__ bool refine_threshold(const uint32_t* __restrict__ arr, int nw, const uint32_t* excl,
+                                                 uint32_t bin1, uint32_t krem, LayerSync* ls, uint32_t target,
+                                                 FusedShared& sh, uint32_t* T, uint32_t* r, uint32_t* own_eq,
+                                                 uint32_t* own_gt) {
+  const int tid = threadIdx.x;
+  zero_words(sh.hist_w, kD2Bins);
+  if (tid == 0) sh.cand_count = 0;
+  __syncthreads();
+  for (int wp = tid; wp < (nw >> 1); wp += kFT) {
+    uint32_t e0 = 0, e1 = 0;
+    if (kExcl) { e0 = excl[2 * wp]; e1 = excl[2 * wp + 1]; }
+    walk_pair(arr, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
+      if ((k0 >> kD1Shift) == bin1 && !((e0 >> j) & 1u)) {
+        atomicAdd(&sh.hist_w[(k0 >> 10) & (kD2Bins - 1)], 1u);
+        const uint32_t slot = list_slot(&sh.cand_count);
+        if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k0;
+      }
+      if ((k1 >> kD1Shift) == bin1 && !((e1 >> j) & 1u)) {
+        atomicAdd(&sh.hist_w[(k1 >> 10) & (kD2Bins - 1)], 1u);
+        const uint32_t slot = list_slot(&sh.cand_count);
+        if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k1;
+      }
+    });
+  }
+  __syncthreads();
+  const uint32_t ncand = sh.cand_count;
+  uint32_t prefix = bin1;
+  uint32_t gt = 0;
+  for (int round = 0; round < 2; ++round) {
+    if (round == 1) {
+      zero_words(sh.hist_w, kD2Bins);
+      __syncthreads();
+      if (ncand <= (uint32_t)kCandCap) {
+        for (uint32_t e = tid; e < ncand; e += kFT) {
+          const uint32_t key = sh.cand_key[e];
+          if ((key >> 10) == prefix) atomicAdd(&sh.hist_w[key & (kD2Bins - 1)], 1u);
+        }
+      } else {
+        for (int wp = tid; wp < (nw >> 1); wp += kFT) {
+          uint32_t e0 = 0, e1 = 0;
+          if (kExcl) { e0 = excl[2 * wp]; e1 = excl[2 * wp + 1]; }
+          walk_pair(arr, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
+            if ((k0 >> 10) == prefix && !((e0 >> j) & 1u)) atomicAdd(&sh.hist_w[k0 & (kD2Bins - 1)], 1u);
+            if ((k1 >> 10) == prefix && !((e1 >> j) & 1u)) atomicAdd(&sh.hist_w[k1 & (kD2Bins - 1)], 1u);
+          });
+        }
+      }
+      __syncthreads();
+    }
+    const uint32_t own[2] = {sh.hist_w[2 * tid], sh.hist_w[2 * tid + 1]};
+    uint32_t v[2] = {own[0], own[1]};
+    if (kSync) {
+      uint32_t* gh = round == 0 ? ls->hist2 : ls->hist3;
+      if (own[0]) atomicAdd(&gh[2 * tid], own[0]);
+      if (own[1]) atomicAdd(&gh[2 * tid + 1], own[1]);
+      if (!layer_barrier(&ls->arrive[2 + round], target, sh)) return false;
+      const uint2 x = __ldcg(reinterpret_cast<const uint2*>(gh) + tid);
+      v[0] = x.x;
+      v[1] = x.y;
+    }
+    uint32_t bin;
+    find_bin<2>(v, krem, sh, &bin, &krem);
+    if ((uint32_t)(2 * tid) > bin) gt += own[0];
+    if ((uint32_t)(2 * tid + 1) > bin) gt += own[1];
+    if (round == 1 && (uint32_t)tid == (bin >> 1)) sh.red[2] = own[bin & 1u];
+    prefix = (prefix << 10) | bin;
+  }
+  __syncthreads();
+  *T = prefix;
+  *r = krem;
+  *own_eq = sh.red[2];
+  *own_gt += gt;
+  return true;
+}
+
+// Ordered marking walk over the keys of `arr`: bit (t, j) of out is set iff the entry is not excluded and its key is
+// above T, or equal to T with fewer than r equal (not excluded) entries before it.  `ties` = number of such equal
+// entries; when all of them are taken no ordering is needed.  With kHist the first digit of `other`'s key of every
+// entry left unmarked is counted in hist.  tmp: nw words of scratch.
+template <bool kExcl, bool kHist>
+__device__ __forceinline__ void mark_walk(const uint32_t* __restrict__ arr, const uint32_t* __restrict__ other, int nw,
+                                          const uint32_t* excl, bool any, uint32_t T, uint32_t r, uint32_t ties,
+                                          uint32_t* out, uint32_t* tmp, uint32_t* hist, FusedShared& sh) {
+  const int tid = threadIdx.x;
+  const bool ordered = any && r < ties;
+  if (ordered) {
+    uint32_t carry = 0;
+    for (int base = 0; base < (nw >> 1); base += kFT) {
+      const int wp = base + tid;
+      uint32_t q0 = 0, q1 = 0;
+      if (wp < (nw >> 1)) {
+        uint32_t e0 = 0, e1 = 0;
+        if (kExcl) { e0 = excl[2 * wp]; e1 = excl[2 * wp + 1]; }
+        walk_pair(arr, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
+          q0 += (k0 == T) & !((e0 >> j) & 1u);
+          q1 += (k1 == T) & !((e1 >> j) & 1u);
+        });
+      }
+      uint32_t total;
+      const uint32_t before = carry + block_excl_scan(q0 + q1, sh, &total);
+      if (wp < (nw >> 1)) {
+        tmp[2 * wp] = before;
+        tmp[2 * wp + 1] = before + q0;
+      }
+      carry += total;
+    }
+    __syncthreads();
+  }
+  for (int wp = tid; wp < (nw >> 1); wp += kFT) {
+    uint32_t e0 = 0, e1 = 0;
+    if (kExcl) { e0 = excl[2 * wp]; e1 = excl[2 * wp + 1]; }
+    uint32_t run0 = 0, run1 = 0;
+    if (ordered) { run0 = tmp[2 * wp]; run1 = tmp[2 * wp + 1]; }
+    uint32_t w0 = 0, w1 = 0;
+    auto decide = [&](uint32_t key, uint32_t e, int j, uint32_t& run) -> uint32_t {
+      const uint32_t free_ = !((e >> j) & 1u);
+      const uint32_t eq = (key == T) & free_;
+      const uint32_t take = ordered ? (eq & (run < r)) : eq;
+      run += eq;
+      return any ? (((key > T) & free_) | take) : 0u;
+    };
+    if (kHist) {
+      walk_pair2(arr, other, nw, wp, [&](uint32_t k0, uint32_t k1, uint32_t o0, uint32_t o1, int j) {
+        const uint32_t m0 = decide(k0, e0, j, run0), m1 = decide(k1, e1, j, run1);
+        w0 |= m0 << j;
+        w1 |= m1 << j;
+        if (!m0) atomicAdd(&hist[o0 >> kD1Shift], 1u);
+        if (!m1) atomicAdd(&hist[o1 >> kD1Shift], 1u);
+      });
+    } else {
+      walk_pair(arr, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
+        w0 |= decide(k0, e0, j, run0) << j;
+        w1 |= decide(k1, e1, j, run1) << j;
+      });
+    }
+    out[2 * wp] = w0;
+    out[2 * wp + 1] = w1;
+  }
+  __syncthreads();
+}
+
+// Finishes a selection on a list of candidates that all share the first digit: `hist2` holds the histogram of their
+// second digit (bits 19..10), k = how many of them belong to the selection.  Returns the threshold key T and the
+// index limit for the ties: a candidate is selected iff key > T, or key == T and 0xfffff - index >= tie_limit (the
+// lowest indices win).  scratch: kD2Bins words that may alias hist2.
+__device__ __forceinline__ void finish_on_list(const uint32_t* list_key, const uint32_t* list_idx, uint32_t ncand,
+                                               uint32_t bin1, uint32_t* hist2, uint32_t k, uint32_t* scratch,
+                                               FusedShared& sh, uint32_t* T_out, uint32_t* tie_limit_out) {
+  const int tid = threadIdx.x;
+  uint32_t bin2, bin3, krem;
+  find_bin_d2(hist2, k, sh, &bin2, &krem);
+  const uint32_t prefix22 = (bin1 << 10) | bin2;
+  zero_words(scratch, kD2Bins);
+  __syncthreads();
+  for (uint32_t e = tid; e < ncand; e += kFT) {
+    const uint32_t key = list_key[e];
+    if ((key >> 10) == prefix22) atomicAdd(&scratch[key & (kD2Bins - 1)], 1u);
+  }
+  __syncthreads();
+  find_bin_d2(scratch, krem, sh, &bin3, &krem);
+  const uint32_t T = (prefix22 << 10) | bin3;
+  const uint32_t r = krem, ties = scratch[bin3];
+  __syncthreads();
+  uint32_t tie_limit = 0;
+  if (r < ties) {
+    // the r lowest indices among the ties: two more rounds over the 20-bit key (0xfffff - index)
+    uint32_t pre = 0, kk = r;
     for (int round = 0; round < 2; ++round) {
       const int shift = round == 0 ? 10 : 0;
-      zero_words(hist_w, kD2Bins);
+      zero_words(scratch, kD2Bins);
       __syncthreads();
-      for (int i = tid; i < n; i += kSelThreads) {
-        const uint32_t key = keys[i];
-        if ((key >> (shift + 10)) == prefix) atomicAdd(&hist_w[(key >> shift) & (kD2Bins - 1)], 1u);
-      }
-      __syncthreads();
-      uint32_t v1[1] = {hist_w[tid]};
-      find_bin<1>(v1, krem, sh, &bin, &krem);
-      prefix = (prefix << 10) | bin;
-    }
-    T1 = prefix;
-    r1 = krem;
-  }
-
-  // ordered marking walk: warp q owns the words [q * wpw, (q + 1) * wpw); entries stage 1 leaves feed the first-digit
-  // histogram of c
-  const int wpw = (nwords + kSelWarps - 1) / kSelWarps;
-  const int w0 = min(warp * wpw, nwords), w1 = min(w0 + wpw, nwords);
-  {
-    uint32_t eq_count = 0;
-    if (b1 > 0) {
-      for (int q = w0; q < w1; ++q) {
-        const int i = q * 32 + lane;
-        eq_count += __popc(__ballot_sync(0xffffffffu, i < n && keys[i] == T1));
-      }
-    }
-    if (lane == 0) sh.old.warp_cnt[warp] = eq_count;
-    zero_words(hist_w, kD1Bins);
-    __syncthreads();
-    uint32_t running = 0;
-    for (int q = 0; q < warp; ++q) running += sh.old.warp_cnt[q];
-    for (int q0 = w0; q0 < w1; q0 += 4) {
-      float cv[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = (q0 + u) * 32 + lane;
-        cv[u] = (b2 > 0 && q0 + u < w1 && i < n) ? __ldcg(cg_out + i) : 0.f;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int q = q0 + u;
-        if (q >= w1) break;   // uniform across the warp
-        const int i = q * 32 + lane;
-        const bool valid = i < n;
-        const uint32_t key = valid ? keys[i] : 0u;
-        const bool eq = b1 > 0 && valid && key == T1;
-        const uint32_t eqm = __ballot_sync(0xffffffffu, eq);
-        const bool take = eq && (running + __popc(eqm & ((1u << lane) - 1u)) < r1);
-        const bool in1 = b1 > 0 && valid && (key > T1 || take);
-        const uint32_t word = __ballot_sync(0xffffffffu, in1);
-        if (lane == 0) sel1[q] = word;
-        running += __popc(eqm);
-        if (b2 > 0 && valid && !in1) atomicAdd(&hist_w[order_key(cv[u]) >> kD1Shift], 1u);
-      }
-    }
-    __syncthreads();
-  }
-
-  // ---------------- stage 2: the b2 largest c among the entries stage 1 left ----------------
-  if (b2 > 0) {
-    uint32_t v4[4];
-    {
-      const uint4 x = *reinterpret_cast<const uint4*>(hist_w + 4 * tid);
-      v4[0] = x.x; v4[1] = x.y; v4[2] = x.z; v4[3] = x.w;
-    }
-    uint32_t bin1, krem;
-    find_bin<4>(v4, (uint32_t)b2, sh, &bin1, &krem);
-    zero_words(hist_w, kD2Bins);
-    __syncthreads();
-    // one walk over c: entries above the threshold bin are taken, entries inside it become candidates
-    for (int q0 = w0; q0 < w1; q0 += 4) {
-      float cv[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int i = (q0 + u) * 32 + lane;
-        cv[u] = (q0 + u < w1 && i < n) ? __ldcg(cg_out + i) : 0.f;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int q = q0 + u;
-        if (q >= w1) break;
-        const int i = q * 32 + lane;
-        const bool valid = i < n && !((sel1[q] >> lane) & 1u);
-        const uint32_t kc = order_key(cv[u]);
-        const uint32_t d = kc >> kD1Shift;
-        const uint32_t word = __ballot_sync(0xffffffffu, valid && d > bin1);
-        if (lane == 0) sel2[q] = word;
-        const bool cand = valid && d == bin1;
-        const uint32_t cm = __ballot_sync(0xffffffffu, cand);
-        if (cm) {
-          uint32_t base = 0;
-          if (lane == 0) base = atomicAdd(&sh.cand_count, (uint32_t)__popc(cm));
-          base = __shfl_sync(0xffffffffu, base, 0);
-          if (cand) {
-            const uint32_t slot = base + __popc(cm & ((1u << lane) - 1u));
-            if (slot < (uint32_t)p.cand_cap) {
-              cand_key[slot] = kc;
-              cand_idx[slot] = (uint32_t)i;
-            }
-            atomicAdd(&hist_w[(kc >> 10) & (kD2Bins - 1)], 1u);
-          }
-        }
-      }
-    }
-    __syncthreads();
-    const uint32_t ncand = sh.cand_count;
-    if (ncand > (uint32_t)p.cand_cap) {
-      // more entries share the threshold bin than the list holds: full-array select and walk over c
-      uint32_t T2, r2;
-      radix_select(cg_out, n, sel1, (uint32_t)b2, sh.old, &T2, &r2);
-      mark_selected(cg_out, n, sel1, T2, r2, true, sel2, sh.old);
-    } else {
-      uint32_t bin2, bin3;
-      {
-        uint32_t v1[1] = {hist_w[tid]};
-        find_bin<1>(v1, krem, sh, &bin2, &krem);
-      }
-      zero_words(hist_w, kD2Bins);
-      __syncthreads();
-      for (uint32_t e = tid; e < ncand; e += kSelThreads) {
-        const uint32_t kc = cand_key[e];
-        if (((kc >> 10) & (kD2Bins - 1)) == bin2) atomicAdd(&hist_w[kc & (kD2Bins - 1)], 1u);
+      for (uint32_t e = tid; e < ncand; e += kFT) {
+        if (list_key[e] != T) continue;
+        const uint32_t ik = 0xfffffu - list_idx[e];
+        if (round == 0 || (ik >> 10) == pre) atomicAdd(&scratch[(ik >> shift) & (kD2Bins - 1)], 1u);
       }
       __syncthreads();
-      {
-        uint32_t v1[1] = {hist_w[tid]};
-        find_bin<1>(v1, krem, sh, &bin3, &krem);
-      }
-      const uint32_t T2 = (bin1 << kD1Shift) | (bin2 << 10) | bin3;
-      const uint32_t r2 = krem;                 // how many of the entries equal to T2 are taken
-      const uint32_t ties = hist_w[bin3];
-      uint32_t tie_limit = 0;                   // ties with (0xfffff - index) >= tie_limit are taken
-      if (r2 < ties) {
-        // the r2 lowest indices among the ties: two more rounds over the 20-bit key (0xfffff - index)
-        uint32_t pre = 0, kk = r2;
-        for (int round = 0; round < 2; ++round) {
-          const int shift = round == 0 ? 10 : 0;
-          __syncthreads();   // everyone has read the previous histogram
-          zero_words(hist_w, kD2Bins);
-          __syncthreads();
-          for (uint32_t e = tid; e < ncand; e += kSelThreads) {
-            if (cand_key[e] != T2) continue;
-            const uint32_t ik = 0xfffffu - cand_idx[e];
-            if (round == 0 || (ik >> 10) == pre) atomicAdd(&hist_w[(ik >> shift) & (kD2Bins - 1)], 1u);
-          }
-          __syncthreads();
-          uint32_t v1[1] = {hist_w[tid]};
-          uint32_t binx;
-          find_bin<1>(v1, kk, sh, &binx, &kk);
-          pre = (pre << 10) | binx;
-        }
-        tie_limit = pre;
-      }
-      for (uint32_t e = tid; e < ncand; e += kSelThreads) {
-        const uint32_t kc = cand_key[e], i = cand_idx[e];
-        if (kc > T2 || (kc == T2 && 0xfffffu - i >= tie_limit)) atomicOr(&sel2[i >> 5], 1u << (i & 31));
-      }
-      __syncthreads();
+      uint32_t binx;
+      find_bin_d2(scratch, kk, sh, &binx, &kk);
+      pre = (pre << 10) | binx;
     }
-  } else {
-    for (int q = w0 + lane; q < w1; q += 32) sel2[q] = 0;
-    __syncthreads();
+    tie_limit = pre;
   }
-
-  // ---------------- output: ascending indices of sel1 | sel2 ----------------
-  uint32_t cnt = 0;
-  for (int q = w0 + lane; q < w1; q += 32) cnt += __popc(sel1[q] | sel2[q]);
-  cnt = __reduce_add_sync(0xffffffffu, cnt);
-  if (lane == 0) sh.old.warp_cnt[warp] = cnt;
-  __syncthreads();
-  uint32_t running = 0;
-  for (int q = 0; q < warp; ++q) running += sh.old.warp_cnt[q];
-  int32_t* idx = p.idx + (long long)b * p.btot + off;
-  uint8_t* stage = p.stage ? p.stage + (long long)b * p.btot + off : nullptr;
-  for (int q = w0; q < w1; ++q) {
-    const uint32_t s1 = sel1[q], word = s1 | sel2[q];
-    if ((word >> lane) & 1u) {
-      const uint32_t pos = running + __popc(word & ((1u << lane) - 1u));
-      idx[pos] = q * 32 + lane;
-      if (stage) stage[pos] = ((s1 >> lane) & 1u) ? 1 : 2;
-    }
-    running += __popc(word);
-  }
-  if (tid == 0) {
-    p.offsets[(long long)b * (p.Hkv + 1) + g] = (int32_t)off;
-    if (g == p.Hkv - 1) p.offsets[(long long)b * (p.Hkv + 1) + p.Hkv] = (int32_t)(off + bud);
-  }
+  *T_out = T;
+  *tie_limit_out = tie_limit;
 }
 
-size_t fused_smem_bytes(int n, int cand_cap) {
-  const size_t fixed = (sizeof(FusedFixed) + 15) / 16 * 16;
-  const size_t nwords = (size_t)(n + 31) / 32;
-  return fixed + (size_t)((n + 3) / 4) * 16 + 2 * nwords * 4 + (size_t)cand_cap * 8;
+template <bool kAdaptive>
+__global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
+  extern __shared__ __align__(16) uint8_t fused_smem[];
+  FusedShared& sh = *reinterpret_cast<FusedShared*>(fused_smem);
+  const int n = p.n, nw = p.nw;
+  uint32_t* sel1 = reinterpret_cast<uint32_t*>(fused_smem + ((sizeof(FusedShared) + 15) / 16) * 16);
+  uint32_t* sel2 = sel1 + nw;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = p.G;
+  const float Gf = (float)G, invG = 1.0f / Gf;
+  const bool pow2 = (G & (G - 1)) == 0;
+  const size_t head_words = (size_t)32 * nw;
+
+  for (long long item = blockIdx.x; item < p.nitems; item += gridDim.x) {
+    const int b = (int)(item / p.Hkv), g = (int)(item % p.Hkv);
+    const long long h0 = (long long)b * p.Hq + (long long)g * G;
+    const int vf = p.valid_from ? p.valid_from[b * p.Hkv + g] : 0;
+    uint32_t* a_t = p.a_t + (size_t)item * head_words;
+    uint32_t* c_t = p.c_t + (size_t)item * head_words;
+    LayerSync* ls = kAdaptive ? reinterpret_cast<LayerSync*>(p.sync + (size_t)b * layer_sync_stride(p.Hkv)) : nullptr;
+
+    __syncthreads();   // the previous item's shared state is no longer read
+    zero_words(sh.hist_a, 2 * kD1Bins);   // hist_a and hist_c
+    __syncthreads();
+
+    // ---------------- reduce: one pass over attn and vnorm ----------------
+    const float* vg_row = p.group_sum ? p.vnorm + ((long long)b * p.Hkv + g) * n : nullptr;
+    if ((n & 3) == 0) {
+      // a warp takes half of a tile of 8 words (64 float4) per step: lane = (word in tile, quad of four entries), so
+      // that the loads use whole 32-byte sectors and the transposed stores fill whole sectors as well
+      const int n4 = n >> 2;
+      const int units = 2 * ((n4 + 63) / 64);
+      for (int u = warp; u < units; u += kFW) {
+        const int word = (u >> 1) * 8 + (lane & 7), quad = (lane >> 3) + 4 * (u & 1);
+        const int i4 = word * 8 + quad;
+        if (i4 >= n4) continue;
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sc[4] = {0.f, 0.f, 0.f, 0.f};
+        for (int q0 = 0; q0 < G; q0 += 4) {
+          float4 pa[4], pv[4];
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (q0 + v < G) {
+              pa[v] = __ldcs(reinterpret_cast<const float4*>(p.attn + (h0 + q0 + v) * n) + i4);
+              if (!p.group_sum) pv[v] = __ldcs(reinterpret_cast<const float4*>(p.vnorm + (h0 + q0 + v) * n) + i4);
+            }
+          }
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (q0 + v < G) {
+              const float a4[4] = {pa[v].x, pa[v].y, pa[v].z, pa[v].w};
+              float v4[4] = {0.f, 0.f, 0.f, 0.f};
+              if (!p.group_sum) { v4[0] = pv[v].x; v4[1] = pv[v].y; v4[2] = pv[v].z; v4[3] = pv[v].w; }
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float prod = __fmul_rn(__fadd_rn(a4[j], p.eps), v4[j]);
+                if (q0 + v == 0) { sa[j] = a4[j]; sc[j] = prod; }
+                else { sa[j] = __fadd_rn(sa[j], a4[j]); sc[j] = __fadd_rn(sc[j], prod); }
+              }
+            }
+          }
+        }
+        float4 vg4 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p.group_sum) vg4 = __ldcs(reinterpret_cast<const float4*>(vg_row) + i4);
+        const float vgs[4] = {vg4.x, vg4.y, vg4.z, vg4.w};
+        uint32_t ka[4], kc[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          finish_entry(sa[j], sc[j], Gf, invG, pow2, p.eps, p.group_sum, vgs[j], 4 * i4 + j, p.protect_from, vf,
+                       &ka[j], &kc[j]);
+          a_t[(size_t)(4 * quad + j) * nw + word] = ka[j];
+          c_t[(size_t)(4 * quad + j) * nw + word] = kc[j];
+        }
+        count_digits4(sh.hist_a, ka);
+        count_digits4(sh.hist_c, kc);
+      }
+    } else {
+      for (int i = tid; i < n; i += kFT) {
+        float sa = 0.f, sc = 0.f;
+        for (int q = 0; q < G; ++q) {
+          const float a1 = p.attn[(h0 + q) * n + i];
+          const float v1 = p.group_sum ? 0.f : p.vnorm[(h0 + q) * n + i];
+          const float prod = __fmul_rn(__fadd_rn(a1, p.eps), v1);
+          if (q == 0) { sa = a1; sc = prod; }
+          else { sa = __fadd_rn(sa, a1); sc = __fadd_rn(sc, prod); }
+        }
+        uint32_t ka, kc;
+        finish_entry(sa, sc, Gf, invG, pow2, p.eps, p.group_sum, p.group_sum ? vg_row[i] : 0.f, i, p.protect_from,
+                     vf, &ka, &kc);
+        a_t[(size_t)(i & 31) * nw + (i >> 5)] = ka;
+        c_t[(size_t)(i & 31) * nw + (i >> 5)] = kc;
+        atomicAdd(&sh.hist_a[ka >> kD1Shift], 1u);
+        atomicAdd(&sh.hist_c[kc >> kD1Shift], 1u);
+      }
+    }
+    // the tail of the last word and the padding words: key 0, below every real key
+    for (int i = n + tid; i < 32 * nw; i += kFT) {
+      a_t[(size_t)(i & 31) * nw + (i >> 5)] = 0u;
+      c_t[(size_t)(i & 31) * nw + (i >> 5)] = 0u;
+    }
+    __syncthreads();
+
+    // ---------------- this head's budget and the start of its segment ----------------
+    long long off = 0, bud = 0;
+    bool clipped = false, failed = false;
+    if (kAdaptive) {
+      if (p.b_adapt > 0) {
+        // flattened top-b_adapt over the keys of every head of the slice
+        const uint32_t Hkv = (uint32_t)p.Hkv;
+        uint32_t* lists = reinterpret_cast<uint32_t*>(ls + 1);
+        for (int e = tid; e < kD1Bins; e += kFT) {
+          const uint32_t v = sh.hist_a[e];
+          if (v) atomicAdd(&ls->hist1[e], v);
+        }
+        failed = !layer_barrier(&ls->arrive[0], Hkv, sh);
+        uint32_t T = 0, r = 0, bin1 = 0, krem1 = 0;
+        if (!failed) {
+          uint32_t v[8];
+          const uint4 x = __ldcg(reinterpret_cast<const uint4*>(ls->hist1) + 2 * tid);
+          const uint4 y = __ldcg(reinterpret_cast<const uint4*>(ls->hist1) + 2 * tid + 1);
+          v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
+          find_bin<8>(v, (uint32_t)p.b_adapt, sh, &bin1, &krem1);
+          uint32_t above = 0;
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            if ((uint32_t)(8 * tid + q) > bin1) above += sh.hist_a[8 * tid + q];
+          above = block_sum(above, sh);
+          // this head's keys of the threshold bin
+          if (tid == 0) sh.cand_count = 0;
+          __syncthreads();
+          for (int wp = tid; wp < (nw >> 1); wp += kFT) {
+            walk_pair(a_t, nw, wp, [&](uint32_t k0, uint32_t k1, int) {
+              if ((k0 >> kD1Shift) == bin1) {
+                const uint32_t slot = list_slot(&sh.cand_count);
+                if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k0;
+              }
+              if ((k1 >> kD1Shift) == bin1) {
+                const uint32_t slot = list_slot(&sh.cand_count);
+                if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k1;
+              }
+            });
+          }
+          __syncthreads();
+          const uint32_t mine = sh.cand_count;
+          if (mine <= (uint32_t)kCandCap) {
+            for (uint32_t e = tid; e < mine; e += kFT) lists[(size_t)g * kCandCap + e] = sh.cand_key[e];
+          }
+          if (tid == 0) {
+            ls->ncand[g] = mine;
+            ls->above[g] = above;
+            if (mine > (uint32_t)kCandCap) atomicOr(&ls->overflow, 1u);
+          }
+          failed = !layer_barrier(&ls->arrive[1], Hkv, sh);
+        }
+        if (!failed && ld_acquire(&ls->overflow) == 0) {
+          // every CTA finishes the selection on the union of the lists
+          zero_words(sh.hist_w, kD2Bins);
+          if (tid < kMaxHeads) { sh.head_cnt[tid][0] = 0; sh.head_cnt[tid][1] = 0; }
+          __syncthreads();
+          for (uint32_t q = 0; q < Hkv; ++q) {
+            const uint32_t cnt = __ldcg(&ls->ncand[q]);
+            for (uint32_t e = tid; e < cnt; e += kFT) {
+              const uint32_t key = __ldcg(&lists[(size_t)q * kCandCap + e]);
+              atomicAdd(&sh.hist_w[(key >> 10) & (kD2Bins - 1)], 1u);
+            }
+          }
+          __syncthreads();
+          uint32_t bin2, bin3, krem;
+          find_bin_d2(sh.hist_w, krem1, sh, &bin2, &krem);
+          const uint32_t prefix22 = (bin1 << 10) | bin2;
+          zero_words(sh.hist_w, kD2Bins);
+          __syncthreads();
+          for (uint32_t q = 0; q < Hkv; ++q) {
+            const uint32_t cnt = __ldcg(&ls->ncand[q]);
+            for (uint32_t e = tid; e < cnt; e += kFT) {
+              const uint32_t key = __ldcg(&lists[(size_t)q * kCandCap + e]);
+              if ((key >> 10) == prefix22) atomicAdd(&sh.hist_w[key & (kD2Bins - 1)], 1u);
+            }
+          }
+          __syncthreads();
+          find_bin_d2(sh.hist_w, krem, sh, &bin3, &krem);
+          T = (prefix22 << 10) | bin3;
+          r = krem;
+          for (uint32_t q = 0; q < Hkv; ++q) {
+            const uint32_t cnt = __ldcg(&ls->ncand[q]);
+            uint32_t gt = 0, eq = 0;
+            for (uint32_t e = tid; e < cnt; e += kFT) {
+              const uint32_t key = __ldcg(&lists[(size_t)q * kCandCap + e]);
+              gt += key > T;
+              eq += key == T;
+            }
+            gt = __reduce_add_sync(0xffffffffu, gt);
+            eq = __reduce_add_sync(0xffffffffu, eq);
+            if (lane == 0) {
+              if (gt) atomicAdd(&sh.head_cnt[q][0], gt);
+              if (eq) atomicAdd(&sh.head_cnt[q][1], eq);
+            }
+          }
+          __syncthreads();
+          uint32_t rem = r;
+          for (int q = 0; q <= g; ++q) {
+            const uint32_t gtq = __ldcg(&ls->above[q]) + sh.head_cnt[q][0];
+            const uint32_t take = min(sh.head_cnt[q][1], rem);
+            const long long bq = min((long long)gtq + take + p.floor_b, (long long)n);
+            rem -= take;
+            if (q < g) off += bq;
+            else bud = bq;
+          }
+        } else if (!failed) {
+          // some list did not fit: two more histogram rounds over the slice, then the per-head counts
+          uint32_t own_eq = 0, own_gt = 0;
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            if ((uint32_t)(8 * tid + q) > bin1) own_gt += sh.hist_a[8 * tid + q];
+          failed = !refine_threshold<false, true>(a_t, nw, nullptr, bin1, krem1, ls, Hkv, sh, &T, &r, &own_eq,
+                                                  &own_gt);
+          if (!failed) {
+            const uint32_t total = block_sum(own_gt, sh);
+            if (tid == 0) {
+              ls->cnt[g][0] = total;
+              ls->cnt[g][1] = own_eq;
+            }
+            failed = !layer_barrier(&ls->arrive[4], Hkv, sh);
+          }
+          if (!failed) {
+            uint32_t rem = r;
+            for (int q = 0; q <= g; ++q) {
+              const uint2 c2 = __ldcg(reinterpret_cast<const uint2*>(&ls->cnt[q][0]));
+              const uint32_t take = min(c2.y, rem);
+              const long long bq = min((long long)c2.x + take + p.floor_b, (long long)n);
+              rem -= take;
+              if (q < g) off += bq;
+              else bud = bq;
+            }
+          }
+        }
+      } else {
+        bud = min((long long)p.floor_b, (long long)n);
+        off = (long long)g * bud;
+      }
+      if (off > p.btot) { off = p.btot; clipped = true; }
+      if (off + bud > p.btot) { bud = p.btot - off; clipped = true; }
+      if (p.budgets_out != nullptr && tid == 0) p.budgets_out[(long long)b * p.Hkv + g] = (int32_t)bud;
+    } else if (p.budgets_in == nullptr) {
+      bud = p.uniform_b;
+      off = (long long)g * bud;
+    } else {
+      const int32_t* bb = p.budgets_in + (long long)b * p.Hkv;
+      for (int q = 0; q < g; ++q) off += min(max((long long)bb[q], 0LL), (long long)n);
+      bud = bb[g];
+      if (bud < 0 || bud > n) { bud = min(max(bud, 0LL), (long long)n); clipped = true; }
+      if (off > p.btot) { off = p.btot; clipped = true; }
+      if (off + bud > p.btot) { bud = p.btot - off; clipped = true; }
+    }
+    if (failed) {   // a barrier ran out: report and stop (the CTAs that wait for this one run out as well)
+      if (tid == 0) atomicExch(p.status, (int)CKV_ETIMEOUT);
+      break;
+    }
+    if (clipped && tid == 0) atomicExch(p.status, (int)CKV_EINVAL);
+    long long b1 = (long long)floor((double)p.alpha * (double)bud);
+    b1 = min(max(b1, 0LL), bud);
+    const long long b2 = bud - b1;
+
+    // ---------------- stage 1: the b1 largest a; first digits of c over the entries it leaves ----------------
+    // The stage-2 threshold lies between the b2-th and the (b1+b2)-th largest c of ALL entries (stage 1 removes at
+    // most b1 of the entries above it), so only the bins between those two need counting; entries above them are
+    // merely counted.
+    uint32_t bin1 = kD1Bins, krem1 = 0;      // b1 == 0: no first digit is above or inside the threshold bin
+    uint32_t c_hi = kD1Bins - 1, c_lo = 0;
+    if (b1 > 0) find_bin_d1(sh.hist_a, (uint32_t)b1, sh, &bin1, &krem1);
+    if (b2 > 0) {
+      uint32_t unused;
+      find_bin_d1(sh.hist_c, (uint32_t)b2, sh, &c_hi, &unused);
+      find_bin_d1(sh.hist_c, (uint32_t)bud, sh, &c_lo, &unused);
+    }
+    zero_words(sh.hist_w, kD1Bins);
+    zero_words(sh.hist_a, kD2Bins);          // from here on: second-digit histogram of the stage-1 candidates
+    if (tid == 0) { sh.cand_count = 0; sh.red[0] = 0; }
+    __syncthreads();
+    uint32_t c_above = 0;                     // entries left by stage 1 whose c lies above bin c_hi
+    auto count_c = [&](uint32_t kc) {
+      const uint32_t dc = kc >> kD1Shift;
+      if (dc > c_hi) ++c_above;
+      else if (dc >= c_lo) atomicAdd(&sh.hist_w[dc], 1u);
+    };
+    for (int wp = tid; wp < (nw >> 1); wp += kFT) {
+      uint32_t w0 = 0, w1 = 0;
+      walk_pair2(a_t, c_t, nw, wp, [&](uint32_t k0, uint32_t k1, uint32_t o0, uint32_t o1, int j) {
+        const uint32_t d0 = k0 >> kD1Shift, d1 = k1 >> kD1Shift;
+        if (d0 > bin1) {
+          w0 |= 1u << j;
+        } else if (d0 == bin1) {
+          atomicAdd(&sh.hist_a[(k0 >> 10) & (kD2Bins - 1)], 1u);
+          const uint32_t slot = list_slot(&sh.cand_count);
+          if (slot < (uint32_t)kCandCap) {
+            sh.cand_key[slot] = k0;
+            sh.cand_idx[slot] = (uint32_t)(64 * wp + j);
+            sh.cand_c[slot] = o0;
+          }
+        } else if (b2 > 0) {
+          count_c(o0);
+        }
+        if (d1 > bin1) {
+          w1 |= 1u << j;
+        } else if (d1 == bin1) {
+          atomicAdd(&sh.hist_a[(k1 >> 10) & (kD2Bins - 1)], 1u);
+          const uint32_t slot = list_slot(&sh.cand_count);
+          if (slot < (uint32_t)kCandCap) {
+            sh.cand_key[slot] = k1;
+            sh.cand_idx[slot] = (uint32_t)(64 * wp + 32 + j);
+            sh.cand_c[slot] = o1;
+          }
+        } else if (b2 > 0) {
+          count_c(o1);
+        }
+      });
+      sel1[2 * wp] = w0;
+      sel1[2 * wp + 1] = w1;
+    }
+    __syncthreads();
+    const uint32_t ncand1 = sh.cand_count;
+    uint32_t k2 = (uint32_t)b2;               // rank of the stage-2 threshold inside hist_w
+    if (ncand1 > (uint32_t)kCandCap) {
+      // the threshold bin of a holds more entries than the list: radix rounds and an ordered walk over the arrays,
+      // with a full first-digit histogram of c
+      uint32_t T1, r1, ties1, unused = 0;
+      refine_threshold<false, false>(a_t, nw, nullptr, bin1, krem1, nullptr, 0u, sh, &T1, &r1, &ties1, &unused);
+      zero_words(sh.hist_w, kD1Bins);
+      __syncthreads();
+      if (b2 > 0)
+        mark_walk<false, true>(a_t, c_t, nw, nullptr, true, T1, r1, ties1, sel1, sel2, sh.hist_w, sh);
+      else
+        mark_walk<false, false>(a_t, nullptr, nw, nullptr, true, T1, r1, ties1, sel1, sel2, nullptr, sh);
+    } else {
+      if (ncand1 > 0) {   // b1 > 0
+        uint32_t T1, tie_limit;
+        finish_on_list(sh.cand_key, sh.cand_idx, ncand1, bin1, sh.hist_a, krem1, sh.hist_a, sh, &T1, &tie_limit);
+        for (uint32_t e = tid; e < ncand1; e += kFT) {
+          const uint32_t key = sh.cand_key[e], i = sh.cand_idx[e];
+          if (key > T1 || (key == T1 && 0xfffffu - i >= tie_limit)) atomicOr(&sel1[i >> 5], 1u << (i & 31));
+          else if (b2 > 0) count_c(sh.cand_c[e]);
+        }
+      }
+      const uint32_t above = block_sum(c_above, sh);   // also orders the bit-mask and histogram updates above
+      k2 = (uint32_t)b2 - above;
+    }
+
+    // ---------------- stage 2: the b2 largest c among the entries stage 1 left ----------------
+    if (b2 > 0) {
+      uint32_t bin2, krem2;
+      find_bin_d1(sh.hist_w, k2, sh, &bin2, &krem2);
+      zero_words(sh.hist_w, kD2Bins);
+      if (tid == 0) sh.cand_count = 0;
+      __syncthreads();
+      // one walk over c: entries above the threshold bin are taken, entries inside it become candidates
+      for (int wp = tid; wp < (nw >> 1); wp += kFT) {
+        const uint32_t e0 = sel1[2 * wp], e1 = sel1[2 * wp + 1];
+        uint32_t w0 = 0, w1 = 0;
+        walk_pair(c_t, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
+          const uint32_t dd0 = k0 >> kD1Shift, dd1 = k1 >> kD1Shift;
+          if (dd0 >= bin2 && !((e0 >> j) & 1u)) {
+            if (dd0 > bin2) {
+              w0 |= 1u << j;
+            } else {
+              atomicAdd(&sh.hist_w[(k0 >> 10) & (kD2Bins - 1)], 1u);
+              const uint32_t slot = list_slot(&sh.cand_count);
+              if (slot < (uint32_t)kCandCap) { sh.cand_key[slot] = k0; sh.cand_idx[slot] = (uint32_t)(64 * wp + j); }
+            }
+          }
+          if (dd1 >= bin2 && !((e1 >> j) & 1u)) {
+            if (dd1 > bin2) {
+              w1 |= 1u << j;
+            } else {
+              atomicAdd(&sh.hist_w[(k1 >> 10) & (kD2Bins - 1)], 1u);
+              const uint32_t slot = list_slot(&sh.cand_count);
+              if (slot < (uint32_t)kCandCap) {
+                sh.cand_key[slot] = k1;
+                sh.cand_idx[slot] = (uint32_t)(64 * wp + 32 + j);
+              }
+            }
+          }
+        });
+        sel2[2 * wp] = w0;
+        sel2[2 * wp + 1] = w1;
+      }
+      __syncthreads();
+      const uint32_t ncand2 = sh.cand_count;
+      if (ncand2 > (uint32_t)kCandCap) {
+        // more entries share the threshold bin than the list holds: radix rounds and an ordered walk over all of c
+        uint32_t T2, r2, ties2, unused = 0;
+        refine_threshold<true, false>(c_t, nw, sel1, bin2, krem2, nullptr, 0u, sh, &T2, &r2, &ties2, &unused);
+        mark_walk<true, false>(c_t, nullptr, nw, sel1, true, T2, r2, ties2, sel2, sh.hist_a, nullptr, sh);
+      } else {
+        uint32_t T2, tie_limit;
+        finish_on_list(sh.cand_key, sh.cand_idx, ncand2, bin2, sh.hist_w, krem2, sh.hist_w, sh, &T2, &tie_limit);
+        for (uint32_t e = tid; e < ncand2; e += kFT) {
+          const uint32_t kc = sh.cand_key[e], i = sh.cand_idx[e];
+          if (kc > T2 || (kc == T2 && 0xfffffu - i >= tie_limit)) atomicOr(&sel2[i >> 5], 1u << (i & 31));
+        }
+        __syncthreads();
+      }
+    } else {
+      for (int q = tid; q < nw; q += kFT) sel2[q] = 0;
+      __syncthreads();
+    }
+
+    // ---------------- output: ascending indices of sel1 | sel2, one word per thread, written in warp-wide runs
+    int32_t* idx = p.idx + (long long)b * p.btot + off;
+    uint8_t* stage = p.stage ? p.stage + (long long)b * p.btot + off : nullptr;
+    uint32_t carry = 0;
+    for (int base = 0; base < nw; base += kFT) {
+      const int q = base + tid;
+      const uint32_t s1 = q < nw ? sel1[q] : 0u;
+      const uint32_t word = q < nw ? (s1 | sel2[q]) : 0u;
+      uint32_t total;
+      const uint32_t pos = carry + block_excl_scan((uint32_t)__popc(word), sh, &total);
+      for (int src = 0; src < 32; ++src) {
+        const uint32_t ws = __shfl_sync(0xffffffffu, word, src);
+        if (ws == 0) continue;   // uniform across the warp
+        const uint32_t ps = __shfl_sync(0xffffffffu, pos, src);
+        const uint32_t ss = __shfl_sync(0xffffffffu, s1, src);
+        if ((ws >> lane) & 1u) {
+          const long long o = (long long)ps + __popc(ws & lanemask_lt());
+          if (o < bud) {
+            idx[o] = (base + warp * 32 + src) * 32 + lane;
+            if (stage) stage[o] = ((ss >> lane) & 1u) ? 1 : 2;
+          }
+        }
+      }
+      carry += total;
+    }
+    if (tid == 0) {
+      p.offsets[(long long)b * (p.Hkv + 1) + g] = (int32_t)off;
+      if (g == p.Hkv - 1) p.offsets[(long long)b * (p.Hkv + 1) + p.Hkv] = (int32_t)(off + bud);
+    }
+  }
 }
 
 }  // namespace
 
+size_t select_sync_bytes(const Dims& d) {
+  return d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE ? (size_t)d.nb * layer_sync_stride(d.Hkv) : 0;
+}
+
 cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                                 int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
-                                int smem_limit, cudaStream_t st, int* launches, int* status_word) {
+                                const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word) {
   const bool adaptive = d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE;
-  if (adaptive && d.Hkv > kMaxCluster) return cudaErrorNotSupported;
-  if (d.n > (1 << 20) - 1) return cudaErrorNotSupported;   // the index tie-break works on 20-bit keys
-  int cap = 4096;
-  while (cap >= 1024 && fused_smem_bytes(d.n, cap) > (size_t)smem_limit) cap >>= 1;
-  if (cap < 1024) return cudaErrorNotSupported;
-  const size_t smem = fused_smem_bytes(d.n, cap);
+  const int nw = (int)(select_head_stride(d.n) / 32);
+  if (nw > kMaxWords || d.Hkv > kMaxHeads) return cudaErrorNotSupported;
+  if (adaptive && ws.sync == nullptr) return cudaErrorNotSupported;
+  const size_t smem = (sizeof(FusedShared) + 15) / 16 * 16 + (size_t)2 * nw * sizeof(uint32_t);
+  if (smem > (size_t)dev.smem_optin) return cudaErrorNotSupported;
 
   FusedArgs p;
   p.attn = attn; p.vnorm = vnorm;
   p.budgets_in = d.budget_mode == CKV_BUDGET_GIVEN ? budgets_in : nullptr;
-  p.c = ws.c; p.budgets_out = adaptive ? ws.budgets : nullptr;
+  p.a_t = reinterpret_cast<uint32_t*>(ws.a);
+  p.c_t = reinterpret_cast<uint32_t*>(ws.c);
+  p.sync = adaptive ? reinterpret_cast<uint8_t*>(ws.sync) : nullptr;
+  p.budgets_out = adaptive ? ws.budgets : nullptr;
   p.idx = idx; p.offsets = offsets; p.stage = stage; p.status = status_word;
   p.valid_from = d.valid_from;
-  p.Hq = d.Hq; p.Hkv = d.Hkv; p.G = d.G; p.n = d.n;
+  p.Hq = d.Hq; p.Hkv = d.Hkv; p.G = d.G; p.n = d.n; p.nw = nw;
   p.group_sum = d.group_sum;
   p.protect_from = d.protect_window ? d.n - d.w : d.n;
-  p.cand_cap = cap;
+  p.nitems = (long long)d.nb * d.Hkv;
   p.uniform_b = d.budget; p.btot = d.btot;
   p.b_adapt = d.budget - (long long)d.Hkv * d.floor_b;
   p.floor_b = (int)d.floor_b;
@@ -538,30 +951,33 @@ cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* v
 
   auto kernel = adaptive ? select_fused_kernel<true> : select_fused_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) {
+  int per_sm = 0;
+  if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kFT, smem);
+  if (e != cudaSuccess || per_sm < 1) {
     (void)cudaGetLastError();
     return cudaErrorNotSupported;
   }
+  // every CTA of the grid is resident (the adaptive allocation waits across CTAs); a slice's heads are handled by
+  // neighbouring CTAs of the same round when the grid is a multiple of Hkv
+  long long grid = (long long)per_sm * dev.sm_count;
+  if (grid > p.nitems) grid = p.nitems;
+  if (adaptive) {
+    grid -= grid % d.Hkv;
+    if (grid < d.Hkv) return cudaErrorNotSupported;
+    // histograms, counters and flags of every slice start at zero (the lists behind them need no clearing)
+    e = cudaMemset2DAsync(ws.sync, layer_sync_stride(d.Hkv), 0, sizeof(LayerSync), (size_t)d.nb, st);
+    if (e != cudaSuccess) return e;
+  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((unsigned)((long long)d.nb * d.Hkv));
-  cfg.blockDim = dim3(kSelThreads);
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kFT);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr;
-  attr.id = cudaLaunchAttributeClusterDimension;
-  attr.val.clusterDim.x = (unsigned)(adaptive ? d.Hkv : 1);
-  attr.val.clusterDim.y = 1;
-  attr.val.clusterDim.z = 1;
+  attr.id = cudaLaunchAttributeCooperative;
+  attr.val.cooperative = adaptive ? 1 : 0;
   cfg.attrs = &attr;
   cfg.numAttrs = 1;
-  if (adaptive) {
-    int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, kernel, &cfg);
-    if (e != cudaSuccess || clusters < 1) {
-      (void)cudaGetLastError();
-      return cudaErrorNotSupported;
-    }
-  }
   e = cudaLaunchKernelEx(&cfg, kernel, p);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();

@@ -1,5 +1,4 @@
-"""Steps 3-4 on the GPU: the single-kernel selection (scores of a head in shared memory) and the multi-kernel selection
-(score arrays in the workspace) against the oracle on identical float32 scores, where every integer decision must
+"""Steps 3-4 on the GPU: the single-kernel selection and the multi-kernel selection against the oracle on identical float32 scores, where every integer decision must
 agree bit for bit (Algorithm 1, stage 1 / stage 2; Algorithm 2, budget allocation)."""
 import numpy as np
 import pytest
@@ -113,10 +112,15 @@ def test_ties_at_the_stage_two_threshold_go_to_the_lower_index():
         _check_against_oracle(P, nu, wl, 1, expect_fused=True)
 
 
-def test_shapes_beyond_shared_memory_use_the_multi_kernel_path():
+def test_long_heads_and_heads_beyond_the_single_kernel_limit():
+    # several words per thread in every walk
     P, nu = _scores(9, 1, 4, 70001)
     wl = small_workload(cfg_id=173, Hq=4, Hkv=2, n=70001, budget_mode="adaptive", budget=14000)
-    _check_against_oracle(P, nu, wl, 2, expect_fused=False)
+    _check_against_oracle(P, nu, wl, 2, expect_fused=True)
+    # more than 4096 words per head: left to the multi-kernel path
+    P, nu = _scores(10, 1, 2, 140003)
+    wl = small_workload(cfg_id=177, Hq=2, Hkv=2, n=140003, budget_mode="adaptive", budget=28000)
+    _check_against_oracle(P, nu, wl, 1, expect_fused=False)
 
 
 @pytest.mark.parametrize("floor", [0.0, 0.3, 1.0])
