@@ -5,20 +5,19 @@
 //   reduce   : a_g, c_g from the group's query heads in the fixed float32 operation order of the selection (see
 //              select.cu), turned into order-preserving integer keys and written to a scratch array in a
 //              word-transposed layout (entry i = 32 t + j lives at [j][t]), so that later walks give every thread
-//              whole 32-entry words with coalesced loads; the 12-bit first-digit histograms of a_g and c_g are built
-//              on the way
-//   budgets  : flattened adaptive allocation over the KV heads of a slice, i.e. over several CTAs: the first-digit
-//              histograms are summed in a per-slice block of global memory, every CTA publishes its keys of the
-//              threshold bin, and each CTA then finishes the selection on the union of those short lists; two
-//              bounded barriers per slice (the launch is cooperative, so all CTAs are resident).  Lists that do not
-//              fit fall back to two more histogram rounds with a barrier each
-//   stage 1  : one walk over a and c marks the entries above the threshold bin, collects the entries inside it
-//              (remaining digits and index tie-break run on that short list) and counts the first digit of c for
-//              the entries stage 1 leaves, restricted to the bins the stage-2 threshold can fall into
-//   stage 2  : one walk over c marks the entries above the threshold bin and collects the entries inside it
-//   output   : ordered compaction of the two bit masks into ascending indices, written in coalesced runs
-// The scratch arrays are re-read from L2 (a once or twice, c twice); two CTAs share an SM.  Every decision is taken on
-// the same integer keys and with the same tie rule as the multi-kernel path: both give identical results.  Scores
+//              whole 32-entry words with coalesced loads; the 12-bit first-digit histogram of a_g is built on the way
+//   budgets  : flattened adaptive allocation over the KV heads of a slice, i.e. over several CTAs: three radix rounds
+//              (12 + 10 + 10 bits) whose histograms are summed in a small per-slice block of global memory; the CTAs
+//              of a slice meet at four bounded barriers (the launch is cooperative, so all of them are resident)
+//   stage 1  : the first round is the histogram already built; the second walks the keys once, also collecting the
+//              keys of the threshold bin; the third runs on that short list; an ordered marking walk (ties to the
+//              lower index) writes the stage-1 bit mask and builds the first-digit histogram of c over the entries
+//              stage 1 leaves
+//   stage 2  : one walk over c marks the entries above the threshold bin and collects the entries inside it; the
+//              remaining digits and the index tie-break run on the list
+//   output   : ordered compaction of the two bit masks into ascending indices
+// The scratch arrays are re-read from L2 (a up to four times, c twice); two CTAs share an SM.  Every decision is taken
+// on the same integer keys and with the same tie rule as the multi-kernel path: both give identical results.  Scores
 // must not be NaN (the padding of the last word uses the key 0, which only a NaN bit pattern maps to).
 #include "ckv_internal.h"
 #include "select_common.cuh"
@@ -35,22 +34,16 @@ constexpr int kCandCap = 2048;                 // keys of a threshold bin kept i
 constexpr int kMaxWords = kD1Bins;             // 32-entry words per head (n <= 131072)
 constexpr int kMaxHeads = 64;
 
-// Per nb slice, zeroed before the launch (adaptive budgets only); followed by Hkv lists of kCandCap keys.
+// Per nb slice, zeroed before the launch (adaptive budgets only).
 struct LayerSync {
   uint32_t hist1[kD1Bins];
   uint32_t hist2[kD2Bins];
   uint32_t hist3[kD2Bins];
-  uint32_t cnt[kMaxHeads][2];   // fallback rounds: keys above / equal to the flattened threshold per KV head
-  uint32_t ncand[kMaxHeads];    // keys of the threshold bin per KV head
-  uint32_t above[kMaxHeads];    // keys in higher bins per KV head
-  uint32_t arrive[8];           // one counter per barrier
-  uint32_t overflow;            // some head's list did not fit
-  uint32_t pad[23];
+  uint32_t cnt[kMaxHeads][2];   // keys above / equal to the flattened threshold per KV head
+  uint32_t arrive[4];           // one counter per barrier
+  uint32_t pad[28];
 };
 static_assert(sizeof(LayerSync) % 16 == 0, "slices of the sync block stay 16-byte aligned");
-__host__ __device__ inline size_t layer_sync_stride(int Hkv) {
-  return sizeof(LayerSync) + (size_t)Hkv * kCandCap * sizeof(uint32_t);
-}
 
 struct FusedArgs {
   const float* attn;
@@ -58,7 +51,7 @@ struct FusedArgs {
   const int32_t* budgets_in;   // given budgets [nb, Hkv] or null
   uint32_t* a_t;               // scratch: keys of a, [nb*Hkv][32][nw]
   uint32_t* c_t;               // scratch: keys of c, same layout
-  uint8_t* sync;               // [nb] blocks of layer_sync_stride(Hkv) bytes (adaptive only)
+  LayerSync* sync;             // [nb] (adaptive only)
   int32_t* budgets_out;        // [nb, Hkv]: the budgets used (adaptive mode), may be null
   int32_t* idx;
   int32_t* offsets;
@@ -74,13 +67,10 @@ struct FusedArgs {
 };
 
 struct FusedShared {
-  uint32_t hist_a[kD1Bins];    // first-digit histogram of a; afterwards scratch (list rounds, tie prefixes)
-  uint32_t hist_c[kD1Bins];    // first-digit histogram of c over all entries
+  uint32_t hist_a[kD1Bins];    // first-digit histogram of a; afterwards scratch (tie prefixes of the stage-2 walk)
   uint32_t hist_w[kD1Bins];    // working histogram
   uint32_t cand_key[kCandCap];
   uint32_t cand_idx[kCandCap];
-  uint32_t cand_c[kCandCap];
-  uint32_t head_cnt[kMaxHeads][2];
   uint32_t wtot[kFW];
   uint32_t res_bin, res_k, cand_count, flag;
   uint32_t red[4];
@@ -286,7 +276,7 @@ __device__ __forceinline__ void walk_pair2(const uint32_t* __restrict__ arr_a, c
 
 // Second and third radix round over the keys of `arr` (entries excluded by `excl` skipped) whose first digit is bin1;
 // the first round's result (bin1, krem) comes from a histogram the caller already has.  With kSync the histograms of
-// the rounds are summed over the CTAs of the slice (barriers arrive[2], arrive[3]).  Returns the threshold key T, how
+// the rounds are summed over the CTAs of the slice (barriers arrive[1], arrive[2]).  Returns the threshold key T, how
 // many of the keys equal to T belong to the top k (r), how many keys equal T in this CTA's array (own_eq), and adds
 // this CTA's keys in higher bins of rounds two and three to *own_gt.  Uses cand_key as list.  false = a barrier
 // timed out.
@@ -346,7 +336,7 @@ __device__ __forceinline__ bool refine_threshold(const uint32_t* __restrict__ ar
       uint32_t* gh = round == 0 ? ls->hist2 : ls->hist3;
       if (own[0]) atomicAdd(&gh[2 * tid], own[0]);
       if (own[1]) atomicAdd(&gh[2 * tid + 1], own[1]);
-      if (!layer_barrier(&ls->arrive[2 + round], target, sh)) return false;
+      if (!layer_barrier(&ls->arrive[1 + round], target, sh)) return false;
       const uint2 x = __ldcg(reinterpret_cast<const uint2*>(gh) + tid);
       v[0] = x.x;
       v[1] = x.y;
@@ -485,7 +475,7 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
   const int n = p.n, nw = p.nw;
   uint32_t* sel1 = reinterpret_cast<uint32_t*>(fused_smem + ((sizeof(FusedShared) + 15) / 16) * 16);
   uint32_t* sel2 = sel1 + nw;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const int G = p.G;
   const float Gf = (float)G, invG = 1.0f / Gf;
   const bool pow2 = (G & (G - 1)) == 0;
@@ -497,23 +487,18 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
     const int vf = p.valid_from ? p.valid_from[b * p.Hkv + g] : 0;
     uint32_t* a_t = p.a_t + (size_t)item * head_words;
     uint32_t* c_t = p.c_t + (size_t)item * head_words;
-    LayerSync* ls = kAdaptive ? reinterpret_cast<LayerSync*>(p.sync + (size_t)b * layer_sync_stride(p.Hkv)) : nullptr;
+    LayerSync* ls = kAdaptive ? p.sync + b : nullptr;
 
     __syncthreads();   // the previous item's shared state is no longer read
-    zero_words(sh.hist_a, 2 * kD1Bins);   // hist_a and hist_c
+    zero_words(sh.hist_a, kD1Bins);
     __syncthreads();
 
     // ---------------- reduce: one pass over attn and vnorm ----------------
     const float* vg_row = p.group_sum ? p.vnorm + ((long long)b * p.Hkv + g) * n : nullptr;
     if ((n & 3) == 0) {
-      // a warp takes half of a tile of 8 words (64 float4) per step: lane = (word in tile, quad of four entries), so
-      // that the loads use whole 32-byte sectors and the transposed stores fill whole sectors as well
       const int n4 = n >> 2;
-      const int units = 2 * ((n4 + 63) / 64);
-      for (int u = warp; u < units; u += kFW) {
-        const int word = (u >> 1) * 8 + (lane & 7), quad = (lane >> 3) + 4 * (u & 1);
-        const int i4 = word * 8 + quad;
-        if (i4 >= n4) continue;
+      for (int i4 = tid; i4 < n4; i4 += kFT) {
+        const int word = i4 >> 3, quad = i4 & 7;
         float sa[4] = {0.f, 0.f, 0.f, 0.f}, sc[4] = {0.f, 0.f, 0.f, 0.f};
         for (int q0 = 0; q0 < G; q0 += 4) {
           float4 pa[4], pv[4];
@@ -551,7 +536,6 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
           c_t[(size_t)(4 * quad + j) * nw + word] = kc[j];
         }
         count_digits4(sh.hist_a, ka);
-        count_digits4(sh.hist_c, kc);
       }
     } else {
       for (int i = tid; i < n; i += kFT) {
@@ -569,7 +553,6 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
         a_t[(size_t)(i & 31) * nw + (i >> 5)] = ka;
         c_t[(size_t)(i & 31) * nw + (i >> 5)] = kc;
         atomicAdd(&sh.hist_a[ka >> kD1Shift], 1u);
-        atomicAdd(&sh.hist_c[kc >> kD1Shift], 1u);
       }
     }
     // the tail of the last word and the padding words: key 0, below every real key
@@ -586,131 +569,42 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
       if (p.b_adapt > 0) {
         // flattened top-b_adapt over the keys of every head of the slice
         const uint32_t Hkv = (uint32_t)p.Hkv;
-        uint32_t* lists = reinterpret_cast<uint32_t*>(ls + 1);
         for (int e = tid; e < kD1Bins; e += kFT) {
           const uint32_t v = sh.hist_a[e];
           if (v) atomicAdd(&ls->hist1[e], v);
         }
         failed = !layer_barrier(&ls->arrive[0], Hkv, sh);
-        uint32_t T = 0, r = 0, bin1 = 0, krem1 = 0;
+        uint32_t T = 0, r = 0, own_eq = 0, own_gt = 0;
         if (!failed) {
           uint32_t v[8];
           const uint4 x = __ldcg(reinterpret_cast<const uint4*>(ls->hist1) + 2 * tid);
           const uint4 y = __ldcg(reinterpret_cast<const uint4*>(ls->hist1) + 2 * tid + 1);
           v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
+          uint32_t bin1, krem1;
           find_bin<8>(v, (uint32_t)p.b_adapt, sh, &bin1, &krem1);
-          uint32_t above = 0;
-#pragma unroll
-          for (int q = 0; q < 8; ++q)
-            if ((uint32_t)(8 * tid + q) > bin1) above += sh.hist_a[8 * tid + q];
-          above = block_sum(above, sh);
-          // this head's keys of the threshold bin
-          if (tid == 0) sh.cand_count = 0;
-          __syncthreads();
-          for (int wp = tid; wp < (nw >> 1); wp += kFT) {
-            walk_pair(a_t, nw, wp, [&](uint32_t k0, uint32_t k1, int) {
-              if ((k0 >> kD1Shift) == bin1) {
-                const uint32_t slot = list_slot(&sh.cand_count);
-                if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k0;
-              }
-              if ((k1 >> kD1Shift) == bin1) {
-                const uint32_t slot = list_slot(&sh.cand_count);
-                if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k1;
-              }
-            });
-          }
-          __syncthreads();
-          const uint32_t mine = sh.cand_count;
-          if (mine <= (uint32_t)kCandCap) {
-            for (uint32_t e = tid; e < mine; e += kFT) lists[(size_t)g * kCandCap + e] = sh.cand_key[e];
-          }
-          if (tid == 0) {
-            ls->ncand[g] = mine;
-            ls->above[g] = above;
-            if (mine > (uint32_t)kCandCap) atomicOr(&ls->overflow, 1u);
-          }
-          failed = !layer_barrier(&ls->arrive[1], Hkv, sh);
-        }
-        if (!failed && ld_acquire(&ls->overflow) == 0) {
-          // every CTA finishes the selection on the union of the lists
-          zero_words(sh.hist_w, kD2Bins);
-          if (tid < kMaxHeads) { sh.head_cnt[tid][0] = 0; sh.head_cnt[tid][1] = 0; }
-          __syncthreads();
-          for (uint32_t q = 0; q < Hkv; ++q) {
-            const uint32_t cnt = __ldcg(&ls->ncand[q]);
-            for (uint32_t e = tid; e < cnt; e += kFT) {
-              const uint32_t key = __ldcg(&lists[(size_t)q * kCandCap + e]);
-              atomicAdd(&sh.hist_w[(key >> 10) & (kD2Bins - 1)], 1u);
-            }
-          }
-          __syncthreads();
-          uint32_t bin2, bin3, krem;
-          find_bin_d2(sh.hist_w, krem1, sh, &bin2, &krem);
-          const uint32_t prefix22 = (bin1 << 10) | bin2;
-          zero_words(sh.hist_w, kD2Bins);
-          __syncthreads();
-          for (uint32_t q = 0; q < Hkv; ++q) {
-            const uint32_t cnt = __ldcg(&ls->ncand[q]);
-            for (uint32_t e = tid; e < cnt; e += kFT) {
-              const uint32_t key = __ldcg(&lists[(size_t)q * kCandCap + e]);
-              if ((key >> 10) == prefix22) atomicAdd(&sh.hist_w[key & (kD2Bins - 1)], 1u);
-            }
-          }
-          __syncthreads();
-          find_bin_d2(sh.hist_w, krem, sh, &bin3, &krem);
-          T = (prefix22 << 10) | bin3;
-          r = krem;
-          for (uint32_t q = 0; q < Hkv; ++q) {
-            const uint32_t cnt = __ldcg(&ls->ncand[q]);
-            uint32_t gt = 0, eq = 0;
-            for (uint32_t e = tid; e < cnt; e += kFT) {
-              const uint32_t key = __ldcg(&lists[(size_t)q * kCandCap + e]);
-              gt += key > T;
-              eq += key == T;
-            }
-            gt = __reduce_add_sync(0xffffffffu, gt);
-            eq = __reduce_add_sync(0xffffffffu, eq);
-            if (lane == 0) {
-              if (gt) atomicAdd(&sh.head_cnt[q][0], gt);
-              if (eq) atomicAdd(&sh.head_cnt[q][1], eq);
-            }
-          }
-          __syncthreads();
-          uint32_t rem = r;
-          for (int q = 0; q <= g; ++q) {
-            const uint32_t gtq = __ldcg(&ls->above[q]) + sh.head_cnt[q][0];
-            const uint32_t take = min(sh.head_cnt[q][1], rem);
-            const long long bq = min((long long)gtq + take + p.floor_b, (long long)n);
-            rem -= take;
-            if (q < g) off += bq;
-            else bud = bq;
-          }
-        } else if (!failed) {
-          // some list did not fit: two more histogram rounds over the slice, then the per-head counts
-          uint32_t own_eq = 0, own_gt = 0;
 #pragma unroll
           for (int q = 0; q < 8; ++q)
             if ((uint32_t)(8 * tid + q) > bin1) own_gt += sh.hist_a[8 * tid + q];
           failed = !refine_threshold<false, true>(a_t, nw, nullptr, bin1, krem1, ls, Hkv, sh, &T, &r, &own_eq,
                                                   &own_gt);
-          if (!failed) {
-            const uint32_t total = block_sum(own_gt, sh);
-            if (tid == 0) {
-              ls->cnt[g][0] = total;
-              ls->cnt[g][1] = own_eq;
-            }
-            failed = !layer_barrier(&ls->arrive[4], Hkv, sh);
+        }
+        if (!failed) {
+          const uint32_t total = block_sum(own_gt, sh);
+          if (tid == 0) {
+            ls->cnt[g][0] = total;
+            ls->cnt[g][1] = own_eq;
           }
-          if (!failed) {
-            uint32_t rem = r;
-            for (int q = 0; q <= g; ++q) {
-              const uint2 c2 = __ldcg(reinterpret_cast<const uint2*>(&ls->cnt[q][0]));
-              const uint32_t take = min(c2.y, rem);
-              const long long bq = min((long long)c2.x + take + p.floor_b, (long long)n);
-              rem -= take;
-              if (q < g) off += bq;
-              else bud = bq;
-            }
+          failed = !layer_barrier(&ls->arrive[3], Hkv, sh);
+        }
+        if (!failed) {
+          uint32_t rem = r;
+          for (int q = 0; q <= g; ++q) {
+            const uint2 c2 = __ldcg(reinterpret_cast<const uint2*>(&ls->cnt[q][0]));
+            const uint32_t take = min(c2.y, rem);
+            const long long bq = min((long long)c2.x + take + p.floor_b, (long long)n);
+            rem -= take;
+            if (q < g) off += bq;
+            else bud = bq;
           }
         }
       } else {
@@ -741,88 +635,19 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
     const long long b2 = bud - b1;
 
     // ---------------- stage 1: the b1 largest a; first digits of c over the entries it leaves ----------------
-    // The stage-2 threshold lies between the b2-th and the (b1+b2)-th largest c of ALL entries (stage 1 removes at
-    // most b1 of the entries above it), so only the bins between those two need counting; entries above them are
-    // merely counted.
-    uint32_t bin1 = kD1Bins, krem1 = 0;      // b1 == 0: no first digit is above or inside the threshold bin
-    uint32_t c_hi = kD1Bins - 1, c_lo = 0;
-    if (b1 > 0) find_bin_d1(sh.hist_a, (uint32_t)b1, sh, &bin1, &krem1);
-    if (b2 > 0) {
-      uint32_t unused;
-      find_bin_d1(sh.hist_c, (uint32_t)b2, sh, &c_hi, &unused);
-      find_bin_d1(sh.hist_c, (uint32_t)bud, sh, &c_lo, &unused);
+    uint32_t T1 = 0, r1 = 0, ties1 = 0;
+    if (b1 > 0) {
+      uint32_t bin1, krem1, unused = 0;
+      find_bin_d1(sh.hist_a, (uint32_t)b1, sh, &bin1, &krem1);
+      refine_threshold<false, false>(a_t, nw, nullptr, bin1, krem1, nullptr, 0u, sh, &T1, &r1, &ties1, &unused);
     }
     zero_words(sh.hist_w, kD1Bins);
-    zero_words(sh.hist_a, kD2Bins);          // from here on: second-digit histogram of the stage-1 candidates
-    if (tid == 0) { sh.cand_count = 0; sh.red[0] = 0; }
     __syncthreads();
-    uint32_t c_above = 0;                     // entries left by stage 1 whose c lies above bin c_hi
-    auto count_c = [&](uint32_t kc) {
-      const uint32_t dc = kc >> kD1Shift;
-      if (dc > c_hi) ++c_above;
-      else if (dc >= c_lo) atomicAdd(&sh.hist_w[dc], 1u);
-    };
-    for (int wp = tid; wp < (nw >> 1); wp += kFT) {
-      uint32_t w0 = 0, w1 = 0;
-      walk_pair2(a_t, c_t, nw, wp, [&](uint32_t k0, uint32_t k1, uint32_t o0, uint32_t o1, int j) {
-        const uint32_t d0 = k0 >> kD1Shift, d1 = k1 >> kD1Shift;
-        if (d0 > bin1) {
-          w0 |= 1u << j;
-        } else if (d0 == bin1) {
-          atomicAdd(&sh.hist_a[(k0 >> 10) & (kD2Bins - 1)], 1u);
-          const uint32_t slot = list_slot(&sh.cand_count);
-          if (slot < (uint32_t)kCandCap) {
-            sh.cand_key[slot] = k0;
-            sh.cand_idx[slot] = (uint32_t)(64 * wp + j);
-            sh.cand_c[slot] = o0;
-          }
-        } else if (b2 > 0) {
-          count_c(o0);
-        }
-        if (d1 > bin1) {
-          w1 |= 1u << j;
-        } else if (d1 == bin1) {
-          atomicAdd(&sh.hist_a[(k1 >> 10) & (kD2Bins - 1)], 1u);
-          const uint32_t slot = list_slot(&sh.cand_count);
-          if (slot < (uint32_t)kCandCap) {
-            sh.cand_key[slot] = k1;
-            sh.cand_idx[slot] = (uint32_t)(64 * wp + 32 + j);
-            sh.cand_c[slot] = o1;
-          }
-        } else if (b2 > 0) {
-          count_c(o1);
-        }
-      });
-      sel1[2 * wp] = w0;
-      sel1[2 * wp + 1] = w1;
-    }
-    __syncthreads();
-    const uint32_t ncand1 = sh.cand_count;
-    uint32_t k2 = (uint32_t)b2;               // rank of the stage-2 threshold inside hist_w
-    if (ncand1 > (uint32_t)kCandCap) {
-      // the threshold bin of a holds more entries than the list: radix rounds and an ordered walk over the arrays,
-      // with a full first-digit histogram of c
-      uint32_t T1, r1, ties1, unused = 0;
-      refine_threshold<false, false>(a_t, nw, nullptr, bin1, krem1, nullptr, 0u, sh, &T1, &r1, &ties1, &unused);
-      zero_words(sh.hist_w, kD1Bins);
-      __syncthreads();
-      if (b2 > 0)
-        mark_walk<false, true>(a_t, c_t, nw, nullptr, true, T1, r1, ties1, sel1, sel2, sh.hist_w, sh);
-      else
-        mark_walk<false, false>(a_t, nullptr, nw, nullptr, true, T1, r1, ties1, sel1, sel2, nullptr, sh);
-    } else {
-      if (ncand1 > 0) {   // b1 > 0
-        uint32_t T1, tie_limit;
-        finish_on_list(sh.cand_key, sh.cand_idx, ncand1, bin1, sh.hist_a, krem1, sh.hist_a, sh, &T1, &tie_limit);
-        for (uint32_t e = tid; e < ncand1; e += kFT) {
-          const uint32_t key = sh.cand_key[e], i = sh.cand_idx[e];
-          if (key > T1 || (key == T1 && 0xfffffu - i >= tie_limit)) atomicOr(&sel1[i >> 5], 1u << (i & 31));
-          else if (b2 > 0) count_c(sh.cand_c[e]);
-        }
-      }
-      const uint32_t above = block_sum(c_above, sh);   // also orders the bit-mask and histogram updates above
-      k2 = (uint32_t)b2 - above;
-    }
+    if (b2 > 0)
+      mark_walk<false, true>(a_t, c_t, nw, nullptr, b1 > 0, T1, r1, ties1, sel1, sel2, sh.hist_w, sh);
+    else
+      mark_walk<false, false>(a_t, nullptr, nw, nullptr, b1 > 0, T1, r1, ties1, sel1, sel2, nullptr, sh);
+    const uint32_t k2 = (uint32_t)b2;
 
     // ---------------- stage 2: the b2 largest c among the entries stage 1 left ----------------
     if (b2 > 0) {
@@ -883,28 +708,24 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
       __syncthreads();
     }
 
-    // ---------------- output: ascending indices of sel1 | sel2, one word per thread, written in warp-wide runs
+    // ---------------- output: ascending indices of sel1 | sel2 ----------------
     int32_t* idx = p.idx + (long long)b * p.btot + off;
     uint8_t* stage = p.stage ? p.stage + (long long)b * p.btot + off : nullptr;
     uint32_t carry = 0;
     for (int base = 0; base < nw; base += kFT) {
       const int q = base + tid;
       const uint32_t s1 = q < nw ? sel1[q] : 0u;
-      const uint32_t word = q < nw ? (s1 | sel2[q]) : 0u;
+      uint32_t word = q < nw ? (s1 | sel2[q]) : 0u;
       uint32_t total;
-      const uint32_t pos = carry + block_excl_scan((uint32_t)__popc(word), sh, &total);
-      for (int src = 0; src < 32; ++src) {
-        const uint32_t ws = __shfl_sync(0xffffffffu, word, src);
-        if (ws == 0) continue;   // uniform across the warp
-        const uint32_t ps = __shfl_sync(0xffffffffu, pos, src);
-        const uint32_t ss = __shfl_sync(0xffffffffu, s1, src);
-        if ((ws >> lane) & 1u) {
-          const long long o = (long long)ps + __popc(ws & lanemask_lt());
-          if (o < bud) {
-            idx[o] = (base + warp * 32 + src) * 32 + lane;
-            if (stage) stage[o] = ((ss >> lane) & 1u) ? 1 : 2;
-          }
+      uint32_t pos = carry + block_excl_scan((uint32_t)__popc(word), sh, &total);
+      while (word) {
+        const int j = __ffs(word) - 1;
+        word &= word - 1;
+        if ((long long)pos < bud) {
+          idx[pos] = q * 32 + j;
+          if (stage) stage[pos] = ((s1 >> j) & 1u) ? 1 : 2;
         }
+        ++pos;
       }
       carry += total;
     }
@@ -918,7 +739,7 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
 }  // namespace
 
 size_t select_sync_bytes(const Dims& d) {
-  return d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE ? (size_t)d.nb * layer_sync_stride(d.Hkv) : 0;
+  return d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE ? (size_t)d.nb * sizeof(LayerSync) : 0;
 }
 
 cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
@@ -936,7 +757,7 @@ cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* v
   p.budgets_in = d.budget_mode == CKV_BUDGET_GIVEN ? budgets_in : nullptr;
   p.a_t = reinterpret_cast<uint32_t*>(ws.a);
   p.c_t = reinterpret_cast<uint32_t*>(ws.c);
-  p.sync = adaptive ? reinterpret_cast<uint8_t*>(ws.sync) : nullptr;
+  p.sync = adaptive ? reinterpret_cast<LayerSync*>(ws.sync) : nullptr;
   p.budgets_out = adaptive ? ws.budgets : nullptr;
   p.idx = idx; p.offsets = offsets; p.stage = stage; p.status = status_word;
   p.valid_from = d.valid_from;
@@ -964,8 +785,8 @@ cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* v
   if (adaptive) {
     grid -= grid % d.Hkv;
     if (grid < d.Hkv) return cudaErrorNotSupported;
-    // histograms, counters and flags of every slice start at zero (the lists behind them need no clearing)
-    e = cudaMemset2DAsync(ws.sync, layer_sync_stride(d.Hkv), 0, sizeof(LayerSync), (size_t)d.nb, st);
+    // histograms and counters of every slice start at zero
+    e = cudaMemsetAsync(ws.sync, 0, select_sync_bytes(d), st);
     if (e != cudaSuccess) return e;
   }
   cudaLaunchConfig_t cfg = {};
