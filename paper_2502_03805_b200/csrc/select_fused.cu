@@ -81,22 +81,6 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ uint32_t lanemask_lt() {
-  uint32_t m;
-  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
-  return m;
-}
-
-// Slot in a list for every calling thread; the threads of a warp that call together share one atomic.
-__device__ __forceinline__ uint32_t list_slot(uint32_t* counter) {
-  const uint32_t m = __activemask();
-  const int leader = __ffs(m) - 1;
-  uint32_t base = 0;
-  if ((int)(threadIdx.x & 31) == leader) base = atomicAdd(counter, (uint32_t)__popc(m));
-  base = __shfl_sync(m, base, leader);
-  return base + __popc(m & lanemask_lt());
-}
-
 // Bin of the k-th largest key in a histogram spread over the CTA: thread t holds bins t*PER .. t*PER+PER-1 (higher
 // bin = larger key).  Returns the bin and k minus the keys in higher bins (all threads).
 template <int PER>
@@ -224,7 +208,9 @@ __device__ __forceinline__ void finish_entry(float sa, float sc, float Gf, float
   *kc = order_key(cv);
 }
 
-// Four consecutive keys into a first-digit histogram: neighbours mostly share a bin, one atomic per run.
+// Four consecutive keys into a first-digit histogram: neighbours mostly share a bin (the scores are max-pooled), one
+// atomic per run.  (Adding up the counts of the lanes of a warp that share a bin first, with a warp match, was
+// measured slower.)
 __device__ __forceinline__ void count_digits4(uint32_t* hist, const uint32_t (&k)[4]) {
   uint32_t cur = k[0] >> kD1Shift, run = 1;
 #pragma unroll
@@ -292,18 +278,25 @@ __device__ __forceinline__ bool refine_threshold(const uint32_t* __restrict__ ar
   for (int wp = tid; wp < (nw >> 1); wp += kFT) {
     uint32_t e0 = 0, e1 = 0;
     if (kExcl) { e0 = excl[2 * wp]; e1 = excl[2 * wp + 1]; }
+    // candidate masks first (no divergence inside the walk), then the few candidates one by one
+    uint32_t c0 = 0, c1 = 0;
     walk_pair(arr, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
-      if ((k0 >> kD1Shift) == bin1 && !((e0 >> j) & 1u)) {
-        atomicAdd(&sh.hist_w[(k0 >> 10) & (kD2Bins - 1)], 1u);
-        const uint32_t slot = list_slot(&sh.cand_count);
-        if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k0;
-      }
-      if ((k1 >> kD1Shift) == bin1 && !((e1 >> j) & 1u)) {
-        atomicAdd(&sh.hist_w[(k1 >> 10) & (kD2Bins - 1)], 1u);
-        const uint32_t slot = list_slot(&sh.cand_count);
-        if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = k1;
-      }
+      c0 |= (uint32_t)((k0 >> kD1Shift) == bin1) << j;
+      c1 |= (uint32_t)((k1 >> kD1Shift) == bin1) << j;
     });
+    c0 &= ~e0;
+    c1 &= ~e1;
+    for (int half = 0; half < 2; ++half) {
+      uint32_t cm = half ? c1 : c0;
+      while (cm) {
+        const int j = __ffs(cm) - 1;
+        cm &= cm - 1;
+        const uint32_t key = __ldcg(arr + (size_t)j * nw + 2 * wp + half);
+        atomicAdd(&sh.hist_w[(key >> 10) & (kD2Bins - 1)], 1u);
+        const uint32_t slot = atomicAdd(&sh.cand_count, 1u);
+        if (slot < (uint32_t)kCandCap) sh.cand_key[slot] = key;
+      }
+    }
   }
   __syncthreads();
   const uint32_t ncand = sh.cand_count;
@@ -660,30 +653,32 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
       for (int wp = tid; wp < (nw >> 1); wp += kFT) {
         const uint32_t e0 = sel1[2 * wp], e1 = sel1[2 * wp + 1];
         uint32_t w0 = 0, w1 = 0;
+        uint32_t c0 = 0, c1 = 0;
         walk_pair(c_t, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
           const uint32_t dd0 = k0 >> kD1Shift, dd1 = k1 >> kD1Shift;
-          if (dd0 >= bin2 && !((e0 >> j) & 1u)) {
-            if (dd0 > bin2) {
-              w0 |= 1u << j;
-            } else {
-              atomicAdd(&sh.hist_w[(k0 >> 10) & (kD2Bins - 1)], 1u);
-              const uint32_t slot = list_slot(&sh.cand_count);
-              if (slot < (uint32_t)kCandCap) { sh.cand_key[slot] = k0; sh.cand_idx[slot] = (uint32_t)(64 * wp + j); }
-            }
-          }
-          if (dd1 >= bin2 && !((e1 >> j) & 1u)) {
-            if (dd1 > bin2) {
-              w1 |= 1u << j;
-            } else {
-              atomicAdd(&sh.hist_w[(k1 >> 10) & (kD2Bins - 1)], 1u);
-              const uint32_t slot = list_slot(&sh.cand_count);
-              if (slot < (uint32_t)kCandCap) {
-                sh.cand_key[slot] = k1;
-                sh.cand_idx[slot] = (uint32_t)(64 * wp + 32 + j);
-              }
-            }
-          }
+          w0 |= (uint32_t)(dd0 > bin2) << j;
+          w1 |= (uint32_t)(dd1 > bin2) << j;
+          c0 |= (uint32_t)(dd0 == bin2) << j;
+          c1 |= (uint32_t)(dd1 == bin2) << j;
         });
+        w0 &= ~e0;
+        w1 &= ~e1;
+        c0 &= ~e0;
+        c1 &= ~e1;
+        for (int half = 0; half < 2; ++half) {
+          uint32_t cm = half ? c1 : c0;
+          while (cm) {
+            const int j = __ffs(cm) - 1;
+            cm &= cm - 1;
+            const uint32_t key = __ldcg(c_t + (size_t)j * nw + 2 * wp + half);
+            atomicAdd(&sh.hist_w[(key >> 10) & (kD2Bins - 1)], 1u);
+            const uint32_t slot = atomicAdd(&sh.cand_count, 1u);
+            if (slot < (uint32_t)kCandCap) {
+              sh.cand_key[slot] = key;
+              sh.cand_idx[slot] = (uint32_t)(64 * wp + 32 * half + j);
+            }
+          }
+        }
         sel2[2 * wp] = w0;
         sel2[2 * wp + 1] = w1;
       }
