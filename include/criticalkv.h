@@ -57,7 +57,9 @@ typedef enum {
   CKV_EALIGN = -3,      /* pointer or stride not 16-byte aligned                              */
   CKV_EWORKSPACE = -4,  /* workspace smaller than criticalkv_workspace_bytes reports          */
   CKV_ECUDA = -5,       /* a CUDA runtime/driver call failed (see criticalkv_last_cuda_error) */
-  CKV_ETIMEOUT = -6     /* a bounded device-side wait ran out (read via criticalkv_device_status) */
+  CKV_ETIMEOUT = -6,    /* a bounded device-side wait ran out (read via criticalkv_device_status) */
+  CKV_EBOUNDS = -7      /* CKV_FLAG_DEBUG_CHECKS: a kernel met an index, offset or count outside its buffer; the
+                           access was skipped (read via criticalkv_device_status)                */
 } criticalkv_status;
 
 typedef enum { CKV_F32 = 0, CKV_BF16 = 1 } criticalkv_dtype;
@@ -81,10 +83,22 @@ enum {
   CKV_FLAG_CTA_PAIR_MMA = 1u << 4, /* bf16 projection norm: use the kernel that pairs two CTAs of a cluster per
                                      MMA (tcgen05 cta_group::2) instead of the default single-CTA kernel.  Same
                                      results bit for bit; measured slower on B200 for head_dim 128              */
-  CKV_FLAG_SELECT_MULTIPASS = 1u << 5 /* criticalkv_select: always run steps 3-4 as separate kernels (group scores,
+  CKV_FLAG_SELECT_MULTIPASS = 1u << 5, /* criticalkv_select: always run steps 3-4 as separate kernels (group scores,
                                      budget allocation, two-stage top-k over score arrays in the workspace) even
                                      when a head's scores fit in shared memory and the single-kernel path applies.
                                      Same results bit for bit                                                   */
+  CKV_FLAG_DEBUG_CHECKS = 1u << 6, /* device-side checks in criticalkv_select, criticalkv_compact and
+                                     criticalkv_gather_positions: every index read from idx / offsets / budgets and
+                                     every output position is tested against the bounds the descriptor implies
+                                     before it is used; a violation skips that access, sets the status word to
+                                     CKV_EBOUNDS and lets the kernel finish (no trap).  Without the flag the same
+                                     accesses are skipped silently.  Meant for bring-up of a caller: the stand-in
+                                     for a memory checker where none can be run                                  */
+  CKV_FLAG_REQUIRE_TENSOR_CORES = 1u << 7 /* criticalkv_score: return CKV_ENOTSUP instead of running the CUDA-core
+                                     kernels when a bf16 problem is outside what the tensor-core kernels take
+                                     (window attention: w in {16, 32, 64, 128, 256} and a layout a tensor map can
+                                     express; they are 20 times faster, so a silent change of path is a
+                                     performance cliff; criticalkv_last_path tells which kernels ran)          */
 };
 
 /* Problem descriptor (plain data, copied by every call). */
@@ -251,7 +265,10 @@ CKV_API int criticalkv_diagnose(criticalkv_handle h, const criticalkv_desc* d, c
  * Self-test of the bounded device-side wait every tensor-core kernel uses: launches one CTA that waits, for at most
  * limit_ns nanoseconds, on a barrier nothing will ever signal.  The kernel must give up, write 0 to *observed_device
  * (a device int; 1 would mean the wait claimed success), set the status word to CKV_ETIMEOUT and end normally.
+ * limit_ns above CKV_SELFTEST_MAX_WAIT_NS (100 ms) is refused with CKV_EINVAL: no wait of this library may hold an SM
+ * for long.
  */
+#define CKV_SELFTEST_MAX_WAIT_NS 100000000ull
 CKV_API int criticalkv_selftest_bounded_wait(criticalkv_handle h, uint64_t limit_ns, int* observed_device,
                                              void* stream);
 

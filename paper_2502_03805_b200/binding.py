@@ -21,6 +21,10 @@ CKV_NORM_L1, CKV_NORM_L2 = 0, 1
 CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM, CKV_FLAG_PROTECT_WINDOW = 1, 2, 4, 8
 CKV_FLAG_CTA_PAIR_MMA = 16
 CKV_FLAG_SELECT_MULTIPASS = 32
+CKV_FLAG_DEBUG_CHECKS = 64
+CKV_FLAG_REQUIRE_TENSOR_CORES = 128
+CKV_EBOUNDS = -7
+CKV_SELFTEST_MAX_WAIT_NS = 100_000_000
 CKV_STATIC_SCRATCH_BYTES = (8 << 20) + (64 << 10)
 
 EXPORTS = ("criticalkv_create", "criticalkv_destroy", "criticalkv_workspace_bytes", "criticalkv_score",

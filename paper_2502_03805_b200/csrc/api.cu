@@ -57,7 +57,8 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (d->reserved != 0 || d->reserved2 != 0) return CKV_EINVAL;
   if (!(d->adaptive_floor >= 0.f && d->adaptive_floor <= 1.f)) return CKV_EINVAL;
   if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM |
-                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_CTA_PAIR_MMA | CKV_FLAG_SELECT_MULTIPASS))
+                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_CTA_PAIR_MMA | CKV_FLAG_SELECT_MULTIPASS |
+                             CKV_FLAG_DEBUG_CHECKS | CKV_FLAG_REQUIRE_TENSOR_CORES))
     return CKV_EINVAL;
   if (d->budget < 0) return CKV_EINVAL;
   if ((long long)d->n * d->Hkv > 0x7fffffffLL) return CKV_ENOTSUP;
@@ -84,6 +85,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   o->group_sum = (d->flags & CKV_FLAG_WO_GROUP_SUM) ? 1 : 0;
   o->protect_window = (d->flags & CKV_FLAG_PROTECT_WINDOW) ? 1 : 0;
   o->norm = d->norm;
+  o->debug_checks = (d->flags & CKV_FLAG_DEBUG_CHECKS) ? 1 : 0;
   o->floor_b = 0;
   if (d->budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
     long long fb = (long long)floor((double)d->adaptive_floor * (double)d->budget / (double)d->Hkv);
@@ -232,6 +234,10 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
                          (float*)(base + L.abar), (void*)(base + L.wsum), (void*)(base + L.gram)};
   int launches = 0, path = 0;
   cudaError_t e = cudaSuccess;
+  if ((d->flags & CKV_FLAG_REQUIRE_TENSOR_CORES) && dd.dtype == CKV_BF16 &&
+      ((d->flags & CKV_FLAG_FORCE_SIMT) || h->cc_major != 10 ||
+       (vnorm && dd.norm == CKV_NORM_L1 && !ckv::vnorm_umma_supported(dd))))
+    return CKV_ENOTSUP;   // nothing has been launched
   if (attn) {
     bool done = false;
     if (dd.dtype == CKV_BF16 && !(d->flags & CKV_FLAG_FORCE_SIMT) && h->cc_major == 10) {
@@ -244,6 +250,7 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
       }
     }
     if (!done && e == cudaSuccess) {
+      if (dd.dtype == CKV_BF16 && (d->flags & CKV_FLAG_REQUIRE_TENSOR_CORES)) return CKV_ENOTSUP;
       e = ckv::launch_window_attn_simt(dd, Qw, K, attn, sw, st, &launches);
       path |= 4;
     }
@@ -278,6 +285,11 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
       }
     }
     if (!done && e == cudaSuccess) {
+      if (dd.dtype == CKV_BF16 && (d->flags & CKV_FLAG_REQUIRE_TENSOR_CORES)) {
+        h->launches += launches;
+        h->last_path = path;
+        return CKV_ENOTSUP;
+      }
       e = ckv::launch_vnorm_simt(dd, V, WO, vnorm, st, &launches);
       path |= 8;
     }
@@ -302,6 +314,8 @@ int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, const float
     return CKV_EALIGN;
   const SelectLayout L = select_layout(dd);
   if (ws_bytes < L.total) return CKV_EWORKSPACE;
+  // heads too long for the single kernel go through the multi-kernel path, whose bit masks live in shared memory
+  if (ckv::two_stage_smem_bytes(dd.n) > (size_t)h->smem_optin) return CKV_ENOTSUP;
   DeviceGuard guard(h->device);
   if (!guard.ok) return CKV_ECUDA;
   char* base = (char*)ws;
@@ -329,7 +343,8 @@ int criticalkv_compact(criticalkv_handle h, const criticalkv_desc* d, const void
   if (!guard.ok) return CKV_ECUDA;
   if (dd.btot == 0) return CKV_OK;
   int launches = 0;
-  cudaError_t e = ckv::launch_compact(dd, K, V, idx, offsets, K_out, V_out, (cudaStream_t)stream, &launches);
+  cudaError_t e = ckv::launch_compact(dd, K, V, idx, offsets, K_out, V_out, h->sm_count, h->status_word,
+                                      (cudaStream_t)stream, &launches);
   h->launches += launches;
   return record_cuda(h, e);
 }
@@ -381,7 +396,8 @@ int criticalkv_gather_positions(criticalkv_handle h, const criticalkv_desc* d, c
   if (!guard.ok) return CKV_ECUDA;
   if (dd.btot == 0) return CKV_OK;
   int launches = 0;
-  cudaError_t e = ckv::launch_gather_positions(dd, pos_in, idx, offsets, pos_out, (cudaStream_t)stream, &launches);
+  cudaError_t e = ckv::launch_gather_positions(dd, pos_in, idx, offsets, pos_out, h->sm_count, h->status_word,
+                                               (cudaStream_t)stream, &launches);
   h->launches += launches;
   return record_cuda(h, e);
 }
@@ -500,12 +516,12 @@ int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc* d, cons
         (e = cudaMemcpyAsync(base + L.V, hv + (size_t)b * L.nV, L.nV, cudaMemcpyHostToDevice, st)) != cudaSuccess ||
         (copy_wo && (e = cudaMemcpyAsync(base + L.WO, hw + (wo_shared ? 0 : (size_t)b * L.nWO), L.nWO,
                                          cudaMemcpyHostToDevice, st)) != cudaSuccess))
-      return record_cuda(h, e);
+      break;   // the common tail below joins the staging streams before the error is returned
     const int32_t* bud = nullptr;
     if (dd.budget_mode == CKV_BUDGET_GIVEN) {
       if ((e = cudaMemcpyAsync(base + L.budgets, budgets_in + (size_t)b * dd.Hkv, (size_t)dd.Hkv * sizeof(int32_t),
                                cudaMemcpyHostToDevice, st)) != cudaSuccess)
-        return record_cuda(h, e);
+        break;
       bud = (const int32_t*)(base + L.budgets);
     }
     rc = criticalkv_score(h, &one, base + L.Qw, base + L.K, base + L.V, base + L.WO, (float*)(base + L.attn),
@@ -526,9 +542,10 @@ int criticalkv_compress_host(criticalkv_handle h, const criticalkv_desc* d, cons
                                          cudaMemcpyDeviceToHost, st)) != cudaSuccess ||
                     (e = cudaMemcpyAsync((char*)V_out + (size_t)b * L.nout, base + L.V_out, L.nout,
                                          cudaMemcpyDeviceToHost, st)) != cudaSuccess)))
-      return record_cuda(h, e);
+      break;
   }
-  // join: the caller's stream continues after both staging streams, and the call returns with the results on the host
+  // join (also after an error: slices already queued keep writing into the caller's host arrays until they finish):
+  // the caller's stream continues after both staging streams, and the call returns with the results on the host
   for (int i = 0; i < 2; ++i) {
     cudaError_t e2 = cudaEventRecord(h->host_event[i], h->host_stream[i]);
     if (e2 == cudaSuccess) e2 = cudaStreamWaitEvent(user, h->host_event[i], 0);
@@ -580,6 +597,7 @@ int criticalkv_diagnose(criticalkv_handle h, const criticalkv_desc* d, const voi
 
 int criticalkv_selftest_bounded_wait(criticalkv_handle h, uint64_t limit_ns, int* observed_device, void* stream) {
   if (!h || !observed_device) return CKV_EINVAL;
+  if (limit_ns > CKV_SELFTEST_MAX_WAIT_NS) return CKV_EINVAL;   // no wait of the library may hold an SM for long
   if (h->cc_major < 9) return CKV_ENOTSUP;
   DeviceGuard guard(h->device);
   if (!guard.ok) return CKV_ECUDA;
@@ -639,6 +657,7 @@ int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc* d, cons
   if (!aligned16(attn) || !aligned16(vnorm) || (reinterpret_cast<uintptr_t>(idx) & 3u) ||
       (reinterpret_cast<uintptr_t>(offsets) & 3u) || (reinterpret_cast<uintptr_t>(budgets_in) & 3u))
     return CKV_EALIGN;
+  if (ckv::two_stage_smem_bytes(dd.n) > (size_t)h->smem_optin) return CKV_ENOTSUP;
   const SelectLayout L = select_layout(dd, false);
   if (L.total > CKV_STATIC_SCRATCH_BYTES) {
     snprintf(h->cuda_error, sizeof(h->cuda_error),
@@ -671,6 +690,7 @@ const char* criticalkv_status_string(int s) {
     case CKV_EWORKSPACE: return "workspace too small";
     case CKV_ECUDA: return "CUDA call failed";
     case CKV_ETIMEOUT: return "device-side wait timed out";
+    case CKV_EBOUNDS: return "debug check: index, offset or count outside its buffer";
     default: return "unknown status";
   }
 }

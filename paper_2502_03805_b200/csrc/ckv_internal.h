@@ -19,6 +19,7 @@ struct Dims {
   int group_sum;      // CKV_FLAG_WO_GROUP_SUM
   int protect_window; // CKV_FLAG_PROTECT_WINDOW
   int norm;           // criticalkv_norm
+  int debug_checks;   // CKV_FLAG_DEBUG_CHECKS
   long long floor_b;  // guaranteed entries per KV head (adaptive budgets)
   long long qs[3], ks[3], vs[3];  // element strides: nb, head, row
   const int32_t* valid_from;      // device [nb, Hkv] or null: first real row of every KV head (rows before it are padding)
@@ -103,9 +104,11 @@ cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* v
                                 int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                                 const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word);
 cudaError_t launch_compact(const Dims& d, const void* K, const void* V, const int32_t* idx, const int32_t* offsets,
-                           void* K_out, void* V_out, cudaStream_t st, int* launches);
+                           void* K_out, void* V_out, int sm_count, int* status_word, cudaStream_t st, int* launches);
 
 cudaError_t launch_gather_positions(const Dims& d, const int32_t* pos_in, const int32_t* idx, const int32_t* offsets,
-                                    int32_t* pos_out, cudaStream_t st, int* launches);
+                                    int32_t* pos_out, int sm_count, int* status_word, cudaStream_t st, int* launches);
+// Dynamic shared memory the multi-kernel two-stage selection needs for a head of n entries.
+size_t two_stage_smem_bytes(int n);
 
 }  // namespace ckv

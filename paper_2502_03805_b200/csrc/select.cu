@@ -66,6 +66,7 @@ struct TwoStageArgs {
   int Hkv, n;
   long long uniform_b, btot;
   float alpha;
+  int debug;   // CKV_FLAG_DEBUG_CHECKS: report a skipped write
 };
 
 __global__ void __launch_bounds__(kSelThreads) two_stage_kernel(TwoStageArgs p) {
@@ -122,8 +123,12 @@ __global__ void __launch_bounds__(kSelThreads) two_stage_kernel(TwoStageArgs p) 
     const uint32_t s1 = sel1[q], word = s1 | sel2[q];
     if ((word >> lane) & 1u) {
       const uint32_t pos = running + __popc(word & ((1u << lane) - 1u));
-      idx[pos] = q * 32 + lane;
-      if (stage) stage[pos] = ((s1 >> lane) & 1u) ? 1 : 2;
+      if ((long long)pos < bud) {   // a selection larger than the budget never writes past the head's segment
+        idx[pos] = q * 32 + lane;
+        if (stage) stage[pos] = ((s1 >> lane) & 1u) ? 1 : 2;
+      } else if (p.debug) {
+        atomicExch(p.status, (int)CKV_EBOUNDS);
+      }
     }
     running += __popc(word);
   }
@@ -291,6 +296,11 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(co
 
 }  // namespace
 
+size_t two_stage_smem_bytes(int n) {
+  // two bit masks of n bits (dynamic) next to the kernel's static histograms
+  return (size_t)2 * ((n + 31) / 32) * sizeof(uint32_t) + sizeof(SelectShared) + 1024;
+}
+
 cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* vnorm, float* a, float* c,
                                 cudaStream_t st, int* launches) {
   dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
@@ -357,6 +367,7 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
   p.a = ws.a; p.c = ws.c; p.budgets = budgets; p.idx = idx; p.offsets = offsets; p.stage = stage;
   p.status = status_word;
   p.Hkv = d.Hkv; p.n = d.n; p.uniform_b = d.budget; p.btot = d.btot; p.alpha = d.alpha;
+  p.debug = d.debug_checks;
   const size_t dyn = (size_t)2 * ((d.n + 31) / 32) * sizeof(uint32_t);
   e = cudaFuncSetAttribute(two_stage_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
   if (e != cudaSuccess) return e;

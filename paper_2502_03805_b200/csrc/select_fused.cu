@@ -60,6 +60,7 @@ struct FusedArgs {
   const int32_t* valid_from;
   int Hq, Hkv, G, n, nw;       // nw: words per head, even
   int group_sum, protect_from;
+  int debug;                   // CKV_FLAG_DEBUG_CHECKS: report a skipped write
   long long nitems;
   long long uniform_b, btot, b_adapt;
   int floor_b;
@@ -716,9 +717,11 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
       while (word) {
         const int j = __ffs(word) - 1;
         word &= word - 1;
-        if ((long long)pos < bud) {
+        if ((long long)pos < bud) {   // a selection larger than the budget never writes past the head's segment
           idx[pos] = q * 32 + j;
           if (stage) stage[pos] = ((s1 >> j) & 1u) ? 1 : 2;
+        } else if (p.debug) {
+          atomicExch(p.status, (int)CKV_EBOUNDS);
         }
         ++pos;
       }
@@ -758,6 +761,7 @@ cudaError_t launch_select_fused(const Dims& d, const float* attn, const float* v
   p.valid_from = d.valid_from;
   p.Hq = d.Hq; p.Hkv = d.Hkv; p.G = d.G; p.n = d.n; p.nw = nw;
   p.group_sum = d.group_sum;
+  p.debug = d.debug_checks;
   p.protect_from = d.protect_window ? d.n - d.w : d.n;
   p.nitems = (long long)d.nb * d.Hkv;
   p.uniform_b = d.budget; p.btot = d.btot;

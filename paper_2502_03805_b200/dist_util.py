@@ -89,9 +89,25 @@ class ShardedCompressor:
         s.score(Qw, K, V, WO, stream=stream)
         local_budgets = None
         if self.adaptive:
-            a_all = self.gather(self.group_scores(stream=stream))
-            B.criticalkv_allocate_budgets(s.handle, self.global_desc, a_all, self.budgets, stream=stream)
-            local_budgets = self.budgets[:, self.g0:self.g1].contiguous()
+            # the gather and the slice are torch operations: they must run on the stream the library calls use,
+            # otherwise they could read the scores or the budgets before the kernels have written them
+            ctx = torch.cuda.stream(stream) if stream is not None and a_is_cuda(self.a_local) else _NullCtx()
+            with ctx:
+                a_all = self.gather(self.group_scores(stream=stream))
+                B.criticalkv_allocate_budgets(s.handle, self.global_desc, a_all, self.budgets, stream=stream)
+                local_budgets = self.budgets[:, self.g0:self.g1].contiguous()
         s.select(budgets_in=local_budgets, stream=stream)
         s.compact(K, V, stream=stream)
         return s
+
+
+class _NullCtx:
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        return False
+
+
+def a_is_cuda(t) -> bool:
+    return bool(getattr(t, "is_cuda", False))

@@ -660,3 +660,37 @@ def test_compress_layer_end_to_end_small():
         seg = out["idx"][g * wl.budget:(g + 1) * wl.budget]
         np.testing.assert_array_equal(out["K_hat"][g * wl.budget:(g + 1) * wl.budget], L.K_store[g][seg])
         np.testing.assert_array_equal(out["V_hat"][g * wl.budget:(g + 1) * wl.budget], L.V_store[g][seg])
+
+
+# ----------------------------------------------------------------------------- equalities between the bounds
+def test_bounds_coincide_where_the_theorems_say_so():
+    r = RNG(77)
+    for trial in range(20):
+        n = int(r.integers(4, 12))
+        A = r.random(n) ** 3
+        A /= A.sum()
+        nu = np.exp(r.standard_normal(n))
+        order = np.argsort(-A)
+        k1 = np.zeros(n, bool)
+        k1[order[: int(r.integers(1, n - 1))]] = True
+        rest = np.flatnonzero(~k1)
+        k2 = np.zeros(n, bool)
+        k2[r.choice(rest, size=int(r.integers(1, rest.size + 1)), replace=False)] = True
+        none = np.zeros(n, bool)
+        # Theorem 3.5 with an empty second stage is Theorem 3.3 for the stage-1 set (sigma is then the kept mass)
+        assert abs(oc.theta_hat_bound(A, nu, k1, none) - oc.theta_bound(A, nu, k1)) < 1e-12
+        # the relaxed bound replaces nu_i of the stage-2 entries by M = min nu: equal when nu is constant
+        flat = np.full(n, float(nu[0]))
+        assert abs(oc.theta_hat_bound(A, flat, k1, k2) - oc.theta_relax_bound(A, flat, k1, k2)) < 1e-12
+        # keeping every entry leaves nothing to perturb
+        assert abs(oc.theta_bound(A, nu, np.ones(n, bool))) < 1e-12
+
+
+def test_bounds_on_a_case_worked_by_hand():
+    # A = (0.5, 0.3, 0.2), nu = (2, 1, 4): C = 1.0 + 0.3 + 0.8 = 2.1.  Stage 1 keeps entries 0 and 1:
+    # sigma = 0.8, 2 - 1/sigma = 0.75, sum of A nu over stage 1 = 1.3.  Stage 2 keeps entry 2 (A nu = 0.8, A = 0.2).
+    A, nu = np.array([0.5, 0.3, 0.2]), np.array([2.0, 1.0, 4.0])
+    k1, k2 = np.array([True, True, False]), np.array([False, False, True])
+    assert abs(oc.theta_hat_bound(A, nu, k1, k2) - (2.1 - 0.75 * 1.3 - 0.75 * 0.8)) < 1e-12       # 0.525
+    assert abs(oc.theta_relax_bound(A, nu, k1, k2) - (2.1 - 0.75 * 1.3 - 1.0 * 0.75 * 0.2)) < 1e-12  # 0.975
+    assert abs(oc.theta_bound(A, nu, k1) - (2.1 - 0.75 * 1.3)) < 1e-12                             # 1.125
