@@ -51,6 +51,13 @@ def all_gather_heads(a_local: torch.Tensor) -> torch.Tensor:
     return torch.cat(parts, dim=1)
 
 
+def local_budget_slice(budgets: torch.Tensor, Hkv: int, world: int, rank: int) -> torch.Tensor:
+    """The columns of budgets[nb, Hkv] (the allocation every rank computes on the gathered scores) that belong to the
+    KV heads of `rank`, as a contiguous [nb, Hkv / world] tensor for criticalkv_select in given-budget mode."""
+    g0, g1 = shard_kv_heads(Hkv, world, rank)
+    return budgets[:, g0:g1].contiguous()
+
+
 class ShardedCompressor:
     """Compression of a layer whose KV heads are split over ranks (a rank holds its KV heads, their query heads and
     their rows of W^O).  Uniform budgets need no communication; flattened adaptive budgets gather the group attention
@@ -62,6 +69,7 @@ class ShardedCompressor:
         from .session import CompressionSession
         self.B = B
         self.g0, self.g1 = shard_kv_heads(Hkv, world, rank)
+        self.Hkv, self.world, self.rank = Hkv, world, rank
         G = Hq // Hkv
         hkv_loc = self.g1 - self.g0
         self.global_desc = B.make_desc(nb=nb, Hq=Hq, Hkv=Hkv, dh=dh, dm=dm, n=n, w=w, pool_k=pool_k, dtype=dtype,
@@ -95,7 +103,7 @@ class ShardedCompressor:
             with ctx:
                 a_all = self.gather(self.group_scores(stream=stream))
                 B.criticalkv_allocate_budgets(s.handle, self.global_desc, a_all, self.budgets, stream=stream)
-                local_budgets = self.budgets[:, self.g0:self.g1].contiguous()
+                local_budgets = local_budget_slice(self.budgets, self.Hkv, self.world, self.rank)
         s.select(budgets_in=local_budgets, stream=stream)
         s.compact(K, V, stream=stream)
         return s

@@ -80,3 +80,46 @@ def test_kv_head_shards_reject_uneven_splits():
 
 def test_single_process_is_identity():
     assert max_over_ranks(3.5) == 3.5
+
+
+def _shard_worker(rank, world, port, out):
+    """One rank of the KV-head-sharded mode on the CPU: its heads' group attention scores go through the real
+    all-gather, the allocation is repeated on the gathered scores, and the rank keeps its slice of the budgets."""
+    import numpy as np
+    import torch
+    from oracle import criticalkv_oracle as oc
+    from paper_2502_03805_b200.dist_util import all_gather_heads, local_budget_slice, shard_kv_heads
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    nb, Hkv, n, btotal = 3, 8, 257, 600
+    a_full = np.random.default_rng(5).random((nb, Hkv, n)).astype(np.float32) ** 4      # same on every rank
+    g0, g1 = shard_kv_heads(Hkv, world, rank)
+    a_all = all_gather_heads(torch.from_numpy(a_full[:, g0:g1].copy()))                  # what the GPU path gathers
+    budgets = torch.tensor(np.stack([oc.allocate_budgets(a_all[b].numpy(), "adaptive", btotal) for b in range(nb)]),
+                           dtype=torch.int32)
+    mine = local_budget_slice(budgets, Hkv, world, rank)
+    out.put((rank, (g0, g1), bool(torch.equal(a_all, torch.from_numpy(a_full))), mine.tolist(), budgets.tolist()))
+    dist.destroy_process_group()
+
+
+def test_sharded_mode_gathers_scores_and_slices_budgets_consistently():
+    import numpy as np
+    from oracle import criticalkv_oracle as oc
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    world = 2
+    procs = [ctx.Process(target=_shard_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    a_full = np.random.default_rng(5).random((3, 8, 257)).astype(np.float32) ** 4
+    want = [oc.allocate_budgets(a_full[b], "adaptive", 600).tolist() for b in range(3)]
+    for rank, (g0, g1), gathered_ok, mine, budgets in res:
+        assert gathered_ok and (g0, g1) == (4 * rank, 4 * rank + 4)
+        assert budgets == want                                   # every rank repeats the same allocation
+        assert mine == [row[g0:g1] for row in want]              # and keeps the columns of its own heads
+    assert all(sum(r0 + r1) == 600 for r0, r1 in zip(res[0][3], res[1][3]))

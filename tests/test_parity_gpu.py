@@ -537,7 +537,7 @@ def test_l2_norm_variant(kw, tensor_cores):
 
 
 @pytest.mark.parametrize("world", [2, 4])
-@pytest.mark.parametrize("variant", ["plain", "group_sum_floor"])
+@pytest.mark.parametrize("variant", ["plain", "group_sum_floor", "side_stream"])
 def test_kv_head_sharded_adaptive_compression_equals_unsharded(world, variant):
     # the ranks of a KV-head-sharded layer are played one after the other on this GPU; the all-gather of the group
     # scores is a concatenation.  Every rank must end up with exactly the rows the unsharded call keeps for its heads.
@@ -562,9 +562,14 @@ def test_kv_head_sharded_adaptive_compression_equals_unsharded(world, variant):
         a_parts.append(sc.group_scores().clone())
         shards.append((sc, t))
     a_all = torch.cat(a_parts, dim=1)
+    # "side_stream": the whole sharded step on a stream that is not torch's current one (the gather and the budget
+    # slice are torch operations and must follow the library calls onto it)
+    side = torch.cuda.Stream() if variant == "side_stream" else None
+    if side is not None:
+        side.wait_stream(torch.cuda.current_stream())
     for sc, t in shards:
         sc.gather = lambda a, a_all=a_all: a_all
-        s = sc.compress(*t)
+        s = sc.compress(*t, stream=side)
         torch.cuda.synchronize()
         assert s.device_status() == 0
         g0, g1 = sc.g0, sc.g1
