@@ -54,8 +54,6 @@ def parse_args():
     p.add_argument("--group-sum", action="store_true",
                    help="measure the grouped-query shortcut of step 2 (CKV_FLAG_WO_GROUP_SUM) instead of the headline path")
     p.add_argument("--l2", action="store_true", help="measure the L2-norm variant of step 2 (CKV_NORM_L2, Gram matrix)")
-    p.add_argument("--cta-pairs", action="store_true",
-                   help="projection norm with two CTAs per MMA (CKV_FLAG_CTA_PAIR_MMA) instead of the default kernel")
     p.add_argument("--select-multipass", action="store_true",
                    help="steps 3-4 as separate kernels (CKV_FLAG_SELECT_MULTIPASS) instead of the single kernel")
     p.add_argument("--shard", default="", choices=["", "kv-heads"],
@@ -343,8 +341,6 @@ def run_mode(args, wl, inputs, rank, world, local, dev):
     nb = wl.layers
     Qw, K, V, WO = (inputs["dev"][k] for k in ("Qw_store", "K_store", "V_store", "WO_store"))
     flags = B.CKV_FLAG_WO_GROUP_SUM if args.group_sum else 0
-    if args.cta_pairs:
-        flags |= B.CKV_FLAG_CTA_PAIR_MMA
     if args.select_multipass:
         flags |= B.CKV_FLAG_SELECT_MULTIPASS
     shard = inputs["shard"]
@@ -469,10 +465,10 @@ def run_mode(args, wl, inputs, rank, world, local, dev):
                         "peak_source": f"{how} (burst bf16 GEMM)", "target": TARGETS["projection_norm"],
                         "peak_sustained": sustained, "frac_of_sustained": achieved / sustained,
                         "ms_per_launch": gemm_avg, "flops_per_launch": work["vnorm_flops"], "traffic": None,
-                        "tensor_core_path": bool(path & 2), "cta_pairs": bool(path & 16)}
+                        "tensor_core_path": bool(path & 2)}
             tr = load_traffic("vnorm_umma_cfg3_traffic.json")
             sh = tr["shape"] if tr else None
-            if (tr and not args.group_sum and not args.l2 and (path & 2) and not (path & 16) and
+            if (tr and not args.group_sum and not args.l2 and (path & 2) and
                     all(sh[k] == v for k, v in (("Hq", wl.Hq), ("Hkv", wl.Hkv), ("head_dim", wl.dh),
                                                 ("d_model", wl.dm), ("n", wl.n)))):
                 roofline["traffic"] = tr["bytes_per_layer"] * nb

@@ -8,7 +8,7 @@
  *
  *   criticalkv_score    steps 1-2   window attention (Algorithm 2) and the projected value-row norm (Algorithm 1)
  *   criticalkv_select   steps 3-4   scores per KV head, budgets, two-stage top-k (Algorithm 1)
- *   criticalkv_compact  step  5     gather of the retained rows (Algorithm 1, "add K_i, V_i to K_hat, V_hat")
+ *   criticalkv_compact  step  5     gather of the retained rows (Algorithm 1, the step that appends the selected entries to the retained cache)
  *
  * Conventions
  *   - Every data pointer is a DEVICE pointer unless the argument is documented as host memory.  The caller owns all
@@ -80,9 +80,6 @@ enum {
                                      c_g = (a_g + eps) * vnorm_g in criticalkv_select.  Hq/Hkv times fewer flops;
                                      not the per-head norm of Algorithm 1 but the norm of the group's summed
                                      projection (the heads of a group share V, so their outputs add in Eq. 2).  */
-  CKV_FLAG_CTA_PAIR_MMA = 1u << 4, /* bf16 projection norm: use the kernel that pairs two CTAs of a cluster per
-                                     MMA (tcgen05 cta_group::2) instead of the default single-CTA kernel.  Same
-                                     results bit for bit; measured slower on B200 for head_dim 128              */
   CKV_FLAG_SELECT_MULTIPASS = 1u << 5, /* criticalkv_select: always run steps 3-4 as separate kernels (group scores,
                                      budget allocation, two-stage top-k over score arrays in the workspace) even
                                      when a head's scores fit in shared memory and the single-kernel path applies.
@@ -281,7 +278,7 @@ CKV_API const char* criticalkv_status_string(int status);
 CKV_API const char* criticalkv_last_cuda_error(criticalkv_handle h);
 /* Which kernels the last criticalkv_score on this handle launched: bit0 tensor-core window attention,
    bit1 tensor-core projection norm, bit2 CUDA-core window attention, bit3 CUDA-core projection norm,
-   bit4 the tensor-core projection norm ran with paired CTAs; bit5: the last criticalkv_select (or
+   bit5: the last criticalkv_select (or
    criticalkv_select_static) ran as the single kernel. */
 CKV_API int criticalkv_last_path(criticalkv_handle h);
 /* Number of kernel launches this handle has issued since it was created. */

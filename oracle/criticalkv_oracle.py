@@ -41,8 +41,8 @@ F32 = np.float32
 
 
 # ----------------------------------------------------------------------------
-# Step 1: observation-window attention (Algorithm 2, steps "Q_hat = Q[-n':]",
-# "A = softmax(Q_hat K^T); A_bar = A.mean(dim=0)", "A_bar = maxpooling(A_bar)";
+# Step 1: observation-window attention (Algorithm 2: the window slice of the queries,
+# the softmax and window-mean step and the max-pooling step;
 # Eq. 2 for the softmax and its scale)
 # ----------------------------------------------------------------------------
 def window_softmax(Qw_h, K_g, scale):
@@ -65,7 +65,7 @@ def window_softmax(Qw_h, K_g, scale):
 
 
 def window_mean(A):
-    """A_bar[i] = (1/w) sum_j A[j, i]  (Algorithm 2: A.mean(dim=0))."""
+    """A_bar[i] = (1/w) sum_j A[j, i]  (Algorithm 2, mean over the window rows)."""
     A = np.asarray(A, dtype=F64)
     return A.sum(axis=0) / F64(A.shape[0])
 
@@ -304,7 +304,7 @@ def select(P, nu, *, G, budget_mode, budget, alpha=0.5, eps=1e-4, budgets_in=Non
 
 
 # ----------------------------------------------------------------------------
-# Step 5: compaction (Algorithm 1: "add K_i, V_i to K_hat, V_hat")
+# Step 5: compaction (Algorithm 1, the steps that append the selected entries to the retained cache)
 # ----------------------------------------------------------------------------
 def compact(K_store, V_store, idx, offsets):
     """Row gather of the stored (unwidened) K, V: [Btot, dh] each, packed like idx."""

@@ -57,7 +57,7 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (d->reserved != 0 || d->reserved2 != 0) return CKV_EINVAL;
   if (!(d->adaptive_floor >= 0.f && d->adaptive_floor <= 1.f)) return CKV_EINVAL;
   if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM |
-                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_CTA_PAIR_MMA | CKV_FLAG_SELECT_MULTIPASS |
+                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_SELECT_MULTIPASS |
                              CKV_FLAG_DEBUG_CHECKS | CKV_FLAG_REQUIRE_TENSOR_CORES))
     return CKV_EINVAL;
   if (d->budget < 0) return CKV_EINVAL;
@@ -270,13 +270,7 @@ int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, const void* 
   } else if (e == cudaSuccess && vnorm) {
     bool done = false;
     if (dd.dtype == CKV_BF16 && !(d->flags & CKV_FLAG_FORCE_SIMT) && h->cc_major == 10) {
-      e = cudaErrorNotSupported;
-      if (d->flags & CKV_FLAG_CTA_PAIR_MMA) {
-        e = ckv::launch_vnorm_umma_pair(dd, V, WO, vnorm, h->sm_count, h->status_word, st, &launches);
-        if (e == cudaSuccess) path |= 16;
-      }
-      if (e == cudaErrorNotSupported)
-        e = ckv::launch_vnorm_umma(dd, V, WO, vnorm, h->sm_count, h->status_word, st, &launches);
+      e = ckv::launch_vnorm_umma(dd, V, WO, vnorm, h->sm_count, h->status_word, st, &launches);
       if (e == cudaSuccess) {
         done = true;
         path |= 2;

@@ -69,8 +69,6 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
 // Tensor-core projection norm (bf16).  cudaErrorNotSupported = this layout cannot be expressed as a tensor map;
 // the caller then uses the CUDA-core kernel.
 bool vnorm_umma_supported(const Dims& d);
-cudaError_t launch_vnorm_umma_pair(const Dims& d, const void* V, const void* WO, float* vnorm, int sm_count,
-                                   int* status_word, cudaStream_t st, int* launches);
 cudaError_t launch_vnorm_umma(const Dims& d, const void* V, const void* WO, float* vnorm, int sm_count,
                               int* status_word, cudaStream_t st, int* launches);
 cudaError_t launch_bounded_wait_selftest(int* status_word, unsigned long long limit_ns, int* observed,

@@ -1,4 +1,4 @@
-// Step 5: compaction of the retained entries (Algorithm 1: "add K_i, V_i to K_hat, V_hat").
+// Step 5: compaction of the retained entries (Algorithm 1, the steps that append the selected entries to the retained cache).
 // K_out[nb, r, :] = K[nb, g, idx[nb, r], :] for every r in head g's segment [offsets[g], offsets[g+1]); same for V.
 // Pure data movement: every row is copied as 16-byte vectors, one lane per vector, consecutive lanes on consecutive
 // vectors of a row (a 256-byte bf16 row of head_dim 128 is 16 lanes), rows of one head read in ascending order.

@@ -122,25 +122,6 @@ def test_forced_cuda_core_path_agrees_with_tensor_core_path():
     pu.check_layer_against_oracle(Ls[0], wl, cc[0])
 
 
-@pytest.mark.parametrize("kw", [
-    dict(n=1500, dm=640, Hq=8, Hkv=2, dh=128),     # ragged token tail (a pair's second tile partly empty), ragged columns
-    dict(n=260, dm=256, Hq=2, Hkv=2, dh=128),      # second CTA's tile almost empty
-    dict(n=1100, dm=192, Hq=4, Hkv=2, dh=64),
-])
-def test_cta_pair_projection_kernel_equals_single_cta_kernel(kw):
-    # both kernels contract a row in the same order inside the tensor core and add the absolute values of the same
-    # columns in the same order, so the opt-in CTA-pair kernel must reproduce the default one bit for bit
-    from paper_2502_03805_b200 import binding as B
-    wl = small_workload(cfg_id=132, dtype="bf16", w=32, kp=7, budget=100, **kw)
-    Ls, single, s1 = _run(wl, layers=(0, 1))
-    _, pair, s2 = _run(wl, layers=(0, 1), flags=B.CKV_FLAG_CTA_PAIR_MMA)
-    assert not (s1.last_path & 16) and s2.last_path & 16
-    for L, a, b in zip(Ls, single, pair):
-        np.testing.assert_array_equal(a["vnorm"], b["vnorm"])
-        np.testing.assert_array_equal(a["idx"], b["idx"])
-        pu.check_layer_against_oracle(L, wl, b)
-
-
 def test_compress_call_can_be_captured_in_a_cuda_graph_and_replayed():
     # the whole path (nine launches, tensor maps passed by value) captured once and replayed on new input contents
     from paper_2502_03805_b200 import session_for, to_device, to_host
