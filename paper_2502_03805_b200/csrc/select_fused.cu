@@ -72,6 +72,7 @@ struct FusedShared {
   uint32_t hist_w[kD1Bins];    // working histogram
   uint32_t cand_key[kCandCap];
   uint32_t cand_idx[kCandCap];
+  uint32_t cand_c[kCandCap];   // stage 1: the c key of every candidate
   uint32_t wtot[kFW];
   uint32_t res_bin, res_k, cand_count, flag;
   uint32_t red[4];
@@ -629,18 +630,77 @@ __global__ void __launch_bounds__(kFT, 2) select_fused_kernel(FusedArgs p) {
     const long long b2 = bud - b1;
 
     // ---------------- stage 1: the b1 largest a; first digits of c over the entries it leaves ----------------
-    uint32_t T1 = 0, r1 = 0, ties1 = 0;
-    if (b1 > 0) {
-      uint32_t bin1, krem1, unused = 0;
-      find_bin_d1(sh.hist_a, (uint32_t)b1, sh, &bin1, &krem1);
-      refine_threshold<false, false>(a_t, nw, nullptr, bin1, krem1, nullptr, 0u, sh, &T1, &r1, &ties1, &unused);
-    }
+    // One walk over a and c: entries above the threshold bin of a are taken, entries inside it are collected (their
+    // remaining digits and the index tie-break run on the list), and the first digit of c is counted for the entries
+    // below it; the candidates that the list rounds reject are counted afterwards.
+    uint32_t bin1 = kD1Bins, krem1 = 0;      // b1 == 0: no first digit is above or inside the threshold bin
+    if (b1 > 0) find_bin_d1(sh.hist_a, (uint32_t)b1, sh, &bin1, &krem1);
     zero_words(sh.hist_w, kD1Bins);
+    zero_words(sh.hist_a, kD2Bins);          // from here on: second-digit histogram of the stage-1 candidates
+    if (tid == 0) sh.cand_count = 0;
     __syncthreads();
-    if (b2 > 0)
-      mark_walk<false, true>(a_t, c_t, nw, nullptr, b1 > 0, T1, r1, ties1, sel1, sel2, sh.hist_w, sh);
-    else
-      mark_walk<false, false>(a_t, nullptr, nw, nullptr, b1 > 0, T1, r1, ties1, sel1, sel2, nullptr, sh);
+    for (int wp = tid; wp < (nw >> 1); wp += kFT) {
+      uint32_t w0 = 0, w1 = 0, c0 = 0, c1 = 0;
+      if (b2 > 0) {
+        walk_pair2(a_t, c_t, nw, wp, [&](uint32_t k0, uint32_t k1, uint32_t o0, uint32_t o1, int j) {
+          const uint32_t d0 = k0 >> kD1Shift, d1 = k1 >> kD1Shift;
+          w0 |= (uint32_t)(d0 > bin1) << j;
+          w1 |= (uint32_t)(d1 > bin1) << j;
+          c0 |= (uint32_t)(d0 == bin1) << j;
+          c1 |= (uint32_t)(d1 == bin1) << j;
+          if (d0 < bin1) atomicAdd(&sh.hist_w[o0 >> kD1Shift], 1u);
+          if (d1 < bin1) atomicAdd(&sh.hist_w[o1 >> kD1Shift], 1u);
+        });
+      } else {
+        walk_pair(a_t, nw, wp, [&](uint32_t k0, uint32_t k1, int j) {
+          const uint32_t d0 = k0 >> kD1Shift, d1 = k1 >> kD1Shift;
+          w0 |= (uint32_t)(d0 > bin1) << j;
+          w1 |= (uint32_t)(d1 > bin1) << j;
+          c0 |= (uint32_t)(d0 == bin1) << j;
+          c1 |= (uint32_t)(d1 == bin1) << j;
+        });
+      }
+      sel1[2 * wp] = w0;
+      sel1[2 * wp + 1] = w1;
+      for (int half = 0; half < 2; ++half) {
+        uint32_t cm = half ? c1 : c0;
+        while (cm) {
+          const int j = __ffs(cm) - 1;
+          cm &= cm - 1;
+          const size_t at = (size_t)j * nw + 2 * wp + half;
+          const uint32_t key = __ldcg(a_t + at);
+          atomicAdd(&sh.hist_a[(key >> 10) & (kD2Bins - 1)], 1u);
+          const uint32_t slot = atomicAdd(&sh.cand_count, 1u);
+          if (slot < (uint32_t)kCandCap) {
+            sh.cand_key[slot] = key;
+            sh.cand_idx[slot] = (uint32_t)(64 * wp + 32 * half + j);
+            sh.cand_c[slot] = b2 > 0 ? __ldcg(c_t + at) : 0u;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    const uint32_t ncand1 = sh.cand_count;
+    if (ncand1 > (uint32_t)kCandCap) {
+      // the threshold bin of a holds more entries than the list: radix rounds and an ordered walk over the arrays
+      uint32_t T1, r1, ties1, unused = 0;
+      refine_threshold<false, false>(a_t, nw, nullptr, bin1, krem1, nullptr, 0u, sh, &T1, &r1, &ties1, &unused);
+      zero_words(sh.hist_w, kD1Bins);
+      __syncthreads();
+      if (b2 > 0)
+        mark_walk<false, true>(a_t, c_t, nw, nullptr, true, T1, r1, ties1, sel1, sel2, sh.hist_w, sh);
+      else
+        mark_walk<false, false>(a_t, nullptr, nw, nullptr, true, T1, r1, ties1, sel1, sel2, nullptr, sh);
+    } else if (ncand1 > 0) {
+      uint32_t T1, tie_limit;
+      finish_on_list(sh.cand_key, sh.cand_idx, ncand1, bin1, sh.hist_a, krem1, sh.hist_a, sh, &T1, &tie_limit);
+      for (uint32_t e = tid; e < ncand1; e += kFT) {
+        const uint32_t key = sh.cand_key[e], i = sh.cand_idx[e];
+        if (key > T1 || (key == T1 && 0xfffffu - i >= tie_limit)) atomicOr(&sel1[i >> 5], 1u << (i & 31));
+        else if (b2 > 0) atomicAdd(&sh.hist_w[sh.cand_c[e] >> kD1Shift], 1u);
+      }
+      __syncthreads();
+    }
     const uint32_t k2 = (uint32_t)b2;
 
     // ---------------- stage 2: the b2 largest c among the entries stage 1 left ----------------

@@ -147,26 +147,46 @@ __global__ void attn_combine_kernel(const float* part_m, const float* part_l, fl
   rowstat[2 * r + 1] = 1.0f / (L * (float)w);
 }
 
-// A CTA pools 1024 consecutive positions of one row from a shared-memory copy (with a halo of (kp-1)/2 on both sides),
-// so every input is read from global memory once.
-constexpr int kPoolTile = 1024;
-__global__ void __launch_bounds__(256) maxpool_kernel(const float* __restrict__ abar, float* __restrict__ attn, int n,
-                                                      int kp) {
-  __shared__ float tile[kPoolTile + 64];
+// A CTA pools 4096 consecutive positions of one row from a shared-memory copy (with a halo of (kp-1)/2 on both sides),
+// so every input is read from global memory once.  The tile is fetched with four 16-byte loads per thread issued
+// before any of them is used; a thread then produces 16 outputs a CTA-width apart, so that neither its shared-memory
+// reads nor its stores conflict.
+constexpr int kPoolTile = 4096;
+constexpr int kPoolThreads = 256;
+__global__ void __launch_bounds__(kPoolThreads) maxpool_kernel(const float* __restrict__ abar, float* __restrict__ attn,
+                                                               int n, int kp) {
+  __shared__ __align__(16) float tile[kPoolTile + 64];   // tile[32 + e] = input i0 + e; halo of at most 31 around it
   const long long base = (long long)blockIdx.y * n;
   const int r = (kp - 1) / 2;          // <= 31
   const int i0 = blockIdx.x * kPoolTile;
-  for (int e = threadIdx.x; e < kPoolTile + 2 * r; e += 256) {
-    const int i = i0 - r + e;
-    tile[e] = (i >= 0 && i < n) ? abar[base + i] : -INFINITY;   // outside the sequence: never the maximum
+  const int tid = threadIdx.x;
+  const float* row = abar + base;
+  if ((n & 3) == 0 && i0 + kPoolTile <= n) {
+    float4 v[kPoolTile / (4 * kPoolThreads)];
+#pragma unroll
+    for (int q = 0; q < kPoolTile / (4 * kPoolThreads); ++q)
+      v[q] = __ldcs(reinterpret_cast<const float4*>(row + i0) + q * kPoolThreads + tid);
+#pragma unroll
+    for (int q = 0; q < kPoolTile / (4 * kPoolThreads); ++q)
+      *reinterpret_cast<float4*>(tile + 32 + 4 * (q * kPoolThreads + tid)) = v[q];
+  } else {
+    for (int e = tid; e < kPoolTile; e += kPoolThreads) {
+      const int i = i0 + e;
+      tile[32 + e] = i < n ? row[i] : -INFINITY;   // outside the sequence: never the maximum
+    }
+  }
+  if (tid < 2 * r) {
+    const int e = tid < r ? tid - r : kPoolTile + (tid - r);
+    const int i = i0 + e;
+    tile[32 + e] = (i >= 0 && i < n) ? row[i] : -INFINITY;
   }
   __syncthreads();
-  for (int e = threadIdx.x; e < kPoolTile; e += 256) {
+  for (int e = tid; e < kPoolTile; e += kPoolThreads) {
     const int i = i0 + e;
     if (i >= n) break;
-    float m = tile[e];
-    for (int k = 1; k <= 2 * r; ++k) m = fmaxf(m, tile[e + k]);
-    attn[base + i] = m;
+    float m = tile[32 + e - r];
+    for (int k = 1; k <= 2 * r; ++k) m = fmaxf(m, tile[32 + e - r + k]);
+    __stcs(attn + base + i, m);
   }
 }
 
@@ -184,7 +204,7 @@ cudaError_t run(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, 
   attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
   k2<<<grid, kThreads, smem, st>>>(a);
   dim3 pgrid((d.n + kPoolTile - 1) / kPoolTile, d.nb * d.Hq);
-  maxpool_kernel<<<pgrid, 256, 0, st>>>(a.abar, attn, d.n, d.kp);
+  maxpool_kernel<<<pgrid, kPoolThreads, 0, st>>>(a.abar, attn, d.n, d.kp);
   *launches += 4;
   return cudaGetLastError();
 }
@@ -228,7 +248,7 @@ cudaError_t launch_attn_combine(const float* part_m, const float* part_l, float*
 
 cudaError_t launch_maxpool(const float* abar, float* attn, int n, int kp, int nrows, cudaStream_t st) {
   dim3 pgrid((n + kPoolTile - 1) / kPoolTile, nrows);
-  maxpool_kernel<<<pgrid, 256, 0, st>>>(abar, attn, n, kp);
+  maxpool_kernel<<<pgrid, kPoolThreads, 0, st>>>(abar, attn, n, kp);
   return cudaGetLastError();
 }
 
