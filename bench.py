@@ -187,7 +187,7 @@ def run_reference(args, wl):
     print(json.dumps(line), flush=True)
 
 
-def parity_check(wl, L, layer, outs, rows_per_head=4096):
+def parity_check(wl, L, layer, outs, rows_per_head=4096, norm="l1"):
     """The timed outputs of one layer against the CPU oracle (outside the timed region): the attention row of every
     query head of one KV group, `rows_per_head` sampled projection norms of every query head, the oracle's selection
     rule applied to the GPU's own float32 scores (must reproduce idx / offsets bit for bit), and the gather against a
@@ -205,7 +205,7 @@ def parity_check(wl, L, layer, outs, rows_per_head=4096):
     group_sum = vnorm.shape[0] == wl.Hkv and wl.Hkv != wl.Hq
     if not group_sum:
         for h in range(wl.Hq):
-            nu = oc.projection_norm(L.V[h // wl.G][None], L.WO[h][None], rows=rows)[0]
+            nu = oc.projection_norm(L.V[h // wl.G][None], L.WO[h][None], rows=rows, norm=norm)[0]
             vnorm_err = max(vnorm_err, float(np.max(np.abs(vnorm[h, rows] - nu) / np.maximum(nu, 1e-30))))
     ref = oc.select(attn, vnorm, G=wl.G, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps,
                     group_sum=group_sum)
@@ -492,7 +492,8 @@ def run_mode(args, wl, inputs, rank, world, local, dev):
                                                "achieved_tflops": atf, "tensor_frac": atf / burst})
             stages["select"]["single_kernel"] = bool(path & 32)
         if inputs["parity_inputs"] is not None:
-            parity = parity_check(wl, inputs["parity_inputs"], inputs["parity_layer"], outs)
+            parity = parity_check(wl, inputs["parity_inputs"], inputs["parity_layer"], outs,
+                                  norm="l2" if args.l2 else "l1")
         cpu = None
         if not args.no_cpu_baseline:
             entries, dt, cores = oracle_sample(wl, 0)
