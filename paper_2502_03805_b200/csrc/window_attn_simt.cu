@@ -153,6 +153,7 @@ __global__ void attn_combine_kernel(const float* part_m, const float* part_l, fl
 // reads nor its stores conflict.
 constexpr int kPoolTile = 4096;
 constexpr int kPoolThreads = 256;
+template <int R>
 __global__ void __launch_bounds__(kPoolThreads) maxpool_kernel(const float* __restrict__ abar, float* __restrict__ attn,
                                                                int n, int kp) {
   __shared__ __align__(16) float tile[kPoolTile + 64];   // tile[32 + e] = input i0 + e; halo of at most 31 around it
@@ -181,12 +182,48 @@ __global__ void __launch_bounds__(kPoolThreads) maxpool_kernel(const float* __re
     tile[32 + e] = (i >= 0 && i < n) ? row[i] : -INFINITY;
   }
   __syncthreads();
+  if (R >= 0 && (n & 3) == 0 && i0 + kPoolTile <= n) {
+    // small kernels (the paper's 7 included): four neighbouring outputs per thread from three 16-byte reads of the
+    // tile, one 16-byte store
+#pragma unroll
+    for (int q = 0; q < kPoolTile / (4 * kPoolThreads); ++q) {
+      const int e = 4 * (q * kPoolThreads + tid);
+      float v[12];
+#pragma unroll
+      for (int u = 0; u < 3; ++u) {
+        const float4 x = *reinterpret_cast<const float4*>(tile + 32 + e - 4 + 4 * u);
+        v[4 * u] = x.x; v[4 * u + 1] = x.y; v[4 * u + 2] = x.z; v[4 * u + 3] = x.w;
+      }
+      float o[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        float m = v[4 + c - (R >= 0 ? R : 0)];
+#pragma unroll
+        for (int k = 1; k <= 2 * (R >= 0 ? R : 0); ++k) m = fmaxf(m, v[4 + c - (R >= 0 ? R : 0) + k]);
+        o[c] = m;
+      }
+      __stcs(reinterpret_cast<float4*>(attn + base + i0 + e), make_float4(o[0], o[1], o[2], o[3]));
+    }
+    return;
+  }
   for (int e = tid; e < kPoolTile; e += kPoolThreads) {
     const int i = i0 + e;
     if (i >= n) break;
     float m = tile[32 + e - r];
     for (int k = 1; k <= 2 * r; ++k) m = fmaxf(m, tile[32 + e - r + k]);
     __stcs(attn + base + i, m);
+  }
+}
+
+// R = (kp - 1) / 2 known at compile time for the small kernels, -1 otherwise
+static void launch_maxpool_kernel(dim3 grid, cudaStream_t st, const float* abar, float* attn, int n, int kp) {
+  switch ((kp - 1) / 2) {
+    case 0: maxpool_kernel<0><<<grid, kPoolThreads, 0, st>>>(abar, attn, n, kp); break;
+    case 1: maxpool_kernel<1><<<grid, kPoolThreads, 0, st>>>(abar, attn, n, kp); break;
+    case 2: maxpool_kernel<2><<<grid, kPoolThreads, 0, st>>>(abar, attn, n, kp); break;
+    case 3: maxpool_kernel<3><<<grid, kPoolThreads, 0, st>>>(abar, attn, n, kp); break;
+    case 4: maxpool_kernel<4><<<grid, kPoolThreads, 0, st>>>(abar, attn, n, kp); break;
+    default: maxpool_kernel<-1><<<grid, kPoolThreads, 0, st>>>(abar, attn, n, kp); break;
   }
 }
 
@@ -204,7 +241,7 @@ cudaError_t run(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, 
   attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
   k2<<<grid, kThreads, smem, st>>>(a);
   dim3 pgrid((d.n + kPoolTile - 1) / kPoolTile, d.nb * d.Hq);
-  maxpool_kernel<<<pgrid, kPoolThreads, 0, st>>>(a.abar, attn, d.n, d.kp);
+  launch_maxpool_kernel(pgrid, st, a.abar, attn, d.n, d.kp);
   *launches += 4;
   return cudaGetLastError();
 }
@@ -248,7 +285,7 @@ cudaError_t launch_attn_combine(const float* part_m, const float* part_l, float*
 
 cudaError_t launch_maxpool(const float* abar, float* attn, int n, int kp, int nrows, cudaStream_t st) {
   dim3 pgrid((n + kPoolTile - 1) / kPoolTile, nrows);
-  maxpool_kernel<<<pgrid, kPoolThreads, 0, st>>>(abar, attn, n, kp);
+  launch_maxpool_kernel(pgrid, st, abar, attn, n, kp);
   return cudaGetLastError();
 }
 
