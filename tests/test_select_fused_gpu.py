@@ -155,3 +155,14 @@ def test_group_summed_scores_on_both_paths():
     for flags, fused in ((B.CKV_FLAG_WO_GROUP_SUM, True),
                          (B.CKV_FLAG_WO_GROUP_SUM | B.CKV_FLAG_SELECT_MULTIPASS, False)):
         _check_against_oracle(P, nu, wl, 4, flags=flags, expect_fused=fused, group_sum=True)
+
+
+@pytest.mark.parametrize("nb,Hkv,G,mode,budget", [(48, 8, 2, "adaptive", 900), (60, 6, 1, "adaptive", 777),
+                                                  (70, 5, 3, "uniform", 101)])
+def test_more_heads_than_resident_ctas(nb, Hkv, G, mode, budget):
+    # more (slice, KV head) items than the GPU holds CTAs of the single kernel: every CTA works on several items, and
+    # the heads of a slice still meet at their barriers (the grid is a multiple of Hkv)
+    n = 700
+    P, nu = _scores(40 + Hkv, nb, Hkv * G, n, pooled=True)
+    wl = small_workload(cfg_id=180 + Hkv, Hq=Hkv * G, Hkv=Hkv, n=n, budget_mode=mode, budget=budget)
+    _check_against_oracle(P, nu, wl, G, expect_fused=True)
