@@ -18,6 +18,20 @@ TIE_BAND = 1e-4
 OUTPUT_RTOL = 1e-3
 
 
+def record_report(name, report):
+    """Appends one JSON line with the parity report of a full-size test to parity_reports.jsonl in the run's output
+    folder (CRITICALKV_REPORT_DIR, or the scratch output folder at the repository root), so that how exact the large
+    comparisons were rests on a record and not on a printed line."""
+    import json
+    import os
+    out_dir = os.environ.get("CRITICALKV_REPORT_DIR") or os.path.join(
+        os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "gpurun_out")
+    os.makedirs(out_dir, exist_ok=True)
+    clean = {k: (v.item() if hasattr(v, "item") else v) for k, v in report.items()}
+    with open(os.path.join(out_dir, "parity_reports.jsonl"), "a") as f:
+        f.write(json.dumps({"test": name, **clean}) + "\n")
+
+
 def rel_err(got, ref):
     got = np.asarray(got, dtype=np.float64)
     ref = np.asarray(ref, dtype=np.float64)

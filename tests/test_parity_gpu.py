@@ -584,7 +584,7 @@ def test_config1_full_parity():
     Ls, outs, s = _run(wl)
     assert (s.last_path & 15) == 3
     rep = pu.check_layer_against_oracle(Ls[0], wl, outs[0])
-    print("config1", rep)
+    pu.record_report("config1 full layer", rep)
 
 
 def test_config2_full_parity():
@@ -592,7 +592,7 @@ def test_config2_full_parity():
     Ls, outs, s = _run(wl)
     assert (s.last_path & 15) == 3
     rep = pu.check_layer_against_oracle(Ls[0], wl, outs[0], full_output_check=True)
-    print("config2", rep)
+    pu.record_report("config2 full layer", rep)
 
 
 def test_config3_two_layers_adaptive_parity():
@@ -604,14 +604,14 @@ def test_config3_two_layers_adaptive_parity():
     assert (s.last_path & 15) == 3
     for L, out in zip(Ls, outs):
         rep = pu.check_layer_against_oracle(L, wl, out)
-        print("config3 layer", L.layer, rep)
+        pu.record_report(f"config3 full layer {L.layer} (share target {L.share_target:.2f})", rep)
 
 
 def test_config3_all_layers_in_one_call_as_benchmarked():
     # the launch configuration the benchmark times: all 32 layers in one call (nb = 32).  Every layer is checked by
     # properties that hold at any size (budgets, ordering, the selection rule applied to the GPU's own float32 scores,
-    # bit-exact gather) and by sampled outputs the oracle computes one by one (one query head's attention row and
-    # 256 projection norms per layer).
+    # bit-exact gather) and by sampled outputs the oracle computes one by one (the attention row of every query head
+    # and 4096 projection norms of every query head, per layer).
     from paper_2502_03805_b200 import session_for, to_device, to_host
     wl = config(3)
     nb, n, G = wl.layers, wl.n, wl.G
@@ -627,11 +627,11 @@ def test_config3_all_layers_in_one_call_as_benchmarked():
         L = make_layer(wl, l)
         for dst, name in ((Qw, "Qw_store"), (K, "K_store"), (V, "V_store"), (WO, "WO_store")):
             dst[l].copy_(to_device(getattr(L, name), "bf16"))
-        h = int(rng.integers(wl.Hq))
-        rows = np.sort(rng.choice(n, 256, replace=False))
-        P_h = oc.max_pool(oc.window_mean(oc.window_softmax(L.Qw[h], L.K[h // G], scale)), wl.kp)
-        nu_h = oc.projection_norm(L.V[h // G][None], L.WO[h][None], rows=rows)[0]
-        expected.append((h, rows, P_h, nu_h))
+        rows = np.sort(rng.choice(n, 4096, replace=False))
+        P_all = np.stack([oc.max_pool(oc.window_mean(oc.window_softmax(L.Qw[h], L.K[h // G], scale)), wl.kp)
+                          for h in range(wl.Hq)])
+        nu_all = oc.projection_norm(L.V, L.WO, rows=rows)
+        expected.append((rows, P_all, nu_all))
         del L
     s = session_for(wl, nb=nb)
     s.compress(Qw, K, V, WO)
@@ -639,11 +639,13 @@ def test_config3_all_layers_in_one_call_as_benchmarked():
     assert s.device_status() == 0 and (s.last_path & 15) == 3
     K16, V16 = K.view(torch.int16), V.view(torch.int16)
     Ko16, Vo16 = s.K_out.view(torch.int16), s.V_out.view(torch.int16)
+    worst_attn = worst_vnorm = 0.0
     for l in range(nb):
-        h, rows, P_h, nu_h = expected[l]
+        rows, P_all, nu_all = expected[l]
         attn, vnorm = to_host(s.attn[l]), to_host(s.vnorm[l])
-        pu.assert_scores_close(attn[h], P_h, f"layer {l} attn head {h}")
-        pu.assert_scores_close(vnorm[h, rows], nu_h, f"layer {l} vnorm head {h} (sampled rows)")
+        worst_attn = max(worst_attn, pu.assert_scores_close(attn, P_all, f"layer {l} attn (all heads)"))
+        worst_vnorm = max(worst_vnorm, pu.assert_scores_close(vnorm[:, rows], nu_all,
+                                                              f"layer {l} vnorm (4096 sampled rows per head)"))
         ref = oc.select(attn, vnorm, G=G, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps)
         off = to_host(s.offsets[l])
         np.testing.assert_array_equal(off, ref["offsets"])
@@ -654,6 +656,10 @@ def test_config3_all_layers_in_one_call_as_benchmarked():
             sel = s.idx[l, off[g]:off[g + 1]].long()
             assert torch.equal(K16[l, g][sel], Ko16[l, off[g]:off[g + 1]])
             assert torch.equal(V16[l, g][sel], Vo16[l, off[g]:off[g + 1]])
+    pu.record_report("config3 all 32 layers in one call", dict(
+        layers=nb, attn_err=worst_attn, attn_heads_per_layer=wl.Hq, vnorm_err=worst_vnorm,
+        vnorm_rows_per_head=4096, selection="oracle rule on the GPU's float32 scores: idx, offsets, stage bit-exact "
+        "on every layer", gather="bit-exact on every head of every layer"))
 
 
 @pytest.mark.parametrize("mode", ["uniform", "adaptive"])
@@ -667,13 +673,16 @@ def test_config4_one_layer_sampled(mode):
     assert (s.last_path & 15) == 3
     L, out = Ls[0], outs[0]
     P = oc.pooled_window_attention(L.Qw, L.K, wl.kp, wl.scale)
-    pu.assert_scores_close(out["attn"], P, "attn")
+    attn_err = pu.assert_scores_close(out["attn"], P, "attn")
     rows = np.sort(np.random.default_rng(4).choice(wl.n, 4096, replace=False))
     nu = oc.projection_norm(L.V, L.WO, rows=rows)
-    pu.assert_scores_close(out["vnorm"][:, rows], nu, "vnorm (sampled rows)")
+    vnorm_err = pu.assert_scores_close(out["vnorm"][:, rows], nu, "vnorm (sampled rows)")
     ref = oc.select(out["attn"], out["vnorm"], G=wl.G, budget_mode=wl.budget_mode, budget=wl.budget,
                     alpha=wl.alpha, eps=wl.eps)
     np.testing.assert_array_equal(out["offsets"], ref["offsets"])
     np.testing.assert_array_equal(out["idx"][: ref["idx"].size], ref["idx"])
     np.testing.assert_array_equal(out["stage"][: ref["idx"].size], ref["stage"])
     pu.assert_compaction_exact(L.K_store, L.V_store, out["idx"], out["offsets"], out["K_out"], out["V_out"])
+    pu.record_report(f"config4 one layer, {mode}", dict(
+        attn_err=attn_err, attn="all 40 heads in full", vnorm_err=vnorm_err, vnorm_rows_per_head=4096,
+        selection="oracle rule on the GPU's float32 scores: idx, offsets, stage bit-exact", gather="bit-exact"))
