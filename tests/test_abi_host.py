@@ -55,6 +55,7 @@ def test_workspace_bytes_are_sane(lib):
     (dict(budget_mode="adaptive", budget=2 * 512 + 1), B.CKV_EINVAL), (dict(budget_mode=9), B.CKV_EINVAL),
     (dict(norm=3), B.CKV_EINVAL), (dict(adaptive_floor=1.5), B.CKV_EINVAL), (dict(adaptive_floor=-0.1), B.CKV_EINVAL), (dict(flags=1 << 8), B.CKV_EINVAL), (dict(flags=1 << 4), B.CKV_EINVAL),
     (dict(k_stride=(0, 0, 63)), B.CKV_EALIGN), (dict(k_stride=(0, 0, 32)), B.CKV_EINVAL),
+    (dict(Hq=65, Hkv=65), B.CKV_ENOTSUP),      # more KV heads per slice than the selection kernels handle
 ])
 def test_bad_descriptors_are_rejected_on_the_host(lib, kw, status):
     assert B.criticalkv_workspace_bytes(_desc(**kw), check=False) == status
