@@ -460,7 +460,9 @@ def run_mode(args, wl, inputs, rank, world, local, dev):
             # the fraction is taken against the burst figure (an upper bound); the kernel is timed inside a long step
             # at the power cap, where the library GEMM behind `bf16_tflops_sustained` runs too: that ratio is given
             # next to it
-            roofline = {"kernel": "projection norm (V W^O row L1 norm), step 2", "bound": "tensor",
+            kernel = ("projection norm (Gram matrix W^O W^O^T and quadratic form per row, L2), step 2" if args.l2 else
+                      "projection norm (V W^O row L1 norm), step 2")
+            roofline = {"kernel": kernel, "bound": "tensor",
                         "achieved": achieved, "peak": burst, "unit": "TFLOP/s", "frac": achieved / burst,
                         "peak_source": f"{how} (burst bf16 GEMM)", "target": TARGETS["projection_norm"],
                         "peak_sustained": sustained, "frac_of_sustained": achieved / sustained,
