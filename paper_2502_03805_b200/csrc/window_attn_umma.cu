@@ -138,6 +138,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
   constexpr int kKSteps = DH / 16;
   constexpr int kPanels = DH / 64;
   const int nsub = PASS == kStats ? a.row_blocks : a.head_groups;
+  const bool flip_tiles = (nsub & 1) == 0;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 2; ++s) {
@@ -231,6 +232,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       uint32_t it_k = 0, item_cnt = 0, t = 0;
+      uint32_t slot_uses[2] = {0, 0};
       for (long long item = blockIdx.x; item < a.nitems && !failed; item += gridDim.x, ++item_cnt) {
         const Item w = decode_item(item, a);
         const int qb = item_cnt % a.qbufs;
@@ -241,8 +243,11 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
           if (!mbar_wait_bounded(k_full(s), (it_k / a.kstages) & 1u, abort_flag)) { failed = true; break; }
           const uint32_t k_addr = sbase + L.k_off + s * L.k_stage;
           for (int sub = 0; sub < nsub; ++sub, ++t) {
-            const uint32_t slot = t & 1u;
-            if (!mbar_wait_bounded(t_empty(slot), ((t >> 1) & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+            // with an even number of sub-tiles per key tile a plain alternation would hand every set the same
+            // sub-tiles for ever (e.g. always the wide head group): the assignment flips from tile to tile
+            const uint32_t slot = (t + (flip_tiles ? it_k : 0u)) & 1u;
+            if (!mbar_wait_bounded(t_empty(slot), (slot_uses[slot] & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+            ++slot_uses[slot];
             tc_fence_after();
             uint32_t idesc, a_addr, b_addr, a_panel, b_panel;
             if (PASS == kStats) {
@@ -292,7 +297,7 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
     const int quad = warp & 3;
     const uint32_t lane_base = tmem_base + ((uint32_t)(quad * 32) << 16) + set * kSlotCols;
     const int first_pos = a.n - W;  // sequence position of window row 0
-    uint32_t item_cnt = 0, t = 0, uses = 0;
+    uint32_t item_cnt = 0, t = 0, uses = 0, tile_cnt = 0;
     for (long long item = blockIdx.x; item < a.nitems && !failed; item += gridDim.x, ++item_cnt) {
       const Item w = decode_item(item, a);
       const int qb = item_cnt % a.qbufs;
@@ -308,13 +313,13 @@ window_attn_umma_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_c
 #pragma unroll
       for (int rb = 0; rb < kMaxRowBlocks; ++rb) { rm[rb] = -INFINITY; rl[rb] = 0.f; }
 
-      for (int kt = w.t0; kt < w.t1 && !failed; ++kt) {
+      for (int kt = w.t0; kt < w.t1 && !failed; ++kt, ++tile_cnt) {
         const int key0 = kt * kKeyTile;
         // some (key, row) pair of this tile is masked: causally (last tiles) or as padding (first tiles)
         const bool tail = key0 + kKeyTile - 1 > first_pos || key0 < vf;
 #pragma unroll 1
         for (int sub = 0; sub < nsub; ++sub, ++t) {
-          if ((t & 1u) != set) continue;
+          if (((t + (flip_tiles ? tile_cnt : 0u)) & 1u) != set) continue;
           if (!__all_sync(0xffffffffu, mbar_wait_bounded(t_full(set), uses & 1u, abort_flag))) { failed = true; break; }
           ++uses;
           tc_fence_after();
@@ -511,8 +516,11 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
   a.subgroups = d.G / Gi;
   a.rows = rows;
   a.row_blocks = (rows + 127) / 128;
-  a.heads_per_group = kSlotCols / d.w < Gi ? kSlotCols / d.w : Gi;
-  a.head_groups = (Gi + a.heads_per_group - 1) / a.heads_per_group;
+  // sweep 2: as few MMAs per key tile as an accumulator slot allows, with the heads spread evenly over them (the two
+  // sets of softmax warps take turns on the sub-tiles)
+  const int max_hpg = kSlotCols / d.w < Gi ? kSlotCols / d.w : Gi;
+  a.head_groups = (Gi + max_hpg - 1) / max_hpg;
+  a.heads_per_group = (Gi + a.head_groups - 1) / a.head_groups;
   a.ntiles = (d.n + kKeyTile - 1) / kKeyTile;
   // enough work items to fill the machine a few times over, but at least 4 key tiles each so that the partial
   // statistics (two per item) fit the workspace sized for one partial per 256 keys
