@@ -45,8 +45,12 @@ SMALL = [
     dict(dtype="bf16", n=1000, w=16, kp=5, budget=77, dh=64, dm=192, Hq=4, Hkv=2),
     dict(dtype="bf16", n=130, w=64, kp=3, budget=40, dh=128, dm=128, Hq=2, Hkv=2),
     dict(dtype="bf16", n=5000, w=32, kp=7, budget_mode="adaptive", budget=2000, dh=128, dm=1024, Hq=16, Hkv=4),
+    # even numbers of sub-tiles per key tile (the sets of softmax warps swap sub-tiles from tile to tile)
+    dict(dtype="bf16", n=2500, w=64, kp=7, budget=200, dh=128, dm=256, Hq=12, Hkv=2),    # sweep 2: 3 + 3 heads
+    dict(dtype="bf16", n=2300, w=32, kp=7, budget=200, dh=128, dm=256, Hq=12, Hkv=2),    # sweep 1: 128 + 64 rows
+    dict(dtype="bf16", n=1900, w=32, kp=5, budget=150, dh=64, dm=128, Hq=16, Hkv=2),     # sweep 1: 128 + 128 rows
 ]
-TENSOR_CORE_CASES = range(12, 17)
+TENSOR_CORE_CASES = range(12, 20)
 
 
 @pytest.mark.parametrize("case", range(len(SMALL)))
