@@ -84,6 +84,13 @@ enum {
                                      budget allocation, two-stage top-k over score arrays in the workspace) even
                                      when a head's scores fit in shared memory and the single-kernel path applies.
                                      Same results bit for bit                                                   */
+  CKV_FLAG_SELECT_SINGLE_KERNEL = 1u << 4, /* criticalkv_select: take the single kernel (one CTA per KV head) also for
+                                     calls with few heads (nb * Hkv at most half the number of SMs), which by
+                                     default run the separate kernels with a thread-block cluster per head: a
+                                     layer at a time that is about twice as fast.  Same results bit for bit      */
+  CKV_FLAG_SELECT_NO_CLUSTER = 1u << 8, /* criticalkv_select: no thread-block clusters in steps 3-4 (the separate
+                                     kernels then give every head one CTA), for contexts where cluster launches are
+                                     not wanted.  Same results bit for bit                                      */
   CKV_FLAG_DEBUG_CHECKS = 1u << 6, /* device-side checks in criticalkv_select, criticalkv_compact and
                                      criticalkv_gather_positions: every index read from idx / offsets / budgets and
                                      every output position is tested against the bounds the descriptor implies
@@ -279,7 +286,7 @@ CKV_API const char* criticalkv_last_cuda_error(criticalkv_handle h);
 /* Which kernels the last criticalkv_score on this handle launched: bit0 tensor-core window attention,
    bit1 tensor-core projection norm, bit2 CUDA-core window attention, bit3 CUDA-core projection norm,
    bit5: the last criticalkv_select (or
-   criticalkv_select_static) ran as the single kernel. */
+   criticalkv_select_static) ran as the single kernel; bit6: its two-stage top-k ran with a cluster per head. */
 CKV_API int criticalkv_last_path(criticalkv_handle h);
 /* Number of kernel launches this handle has issued since it was created. */
 CKV_API int64_t criticalkv_launch_count(criticalkv_handle h);

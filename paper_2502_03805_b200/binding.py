@@ -20,6 +20,8 @@ CKV_BUDGET_UNIFORM, CKV_BUDGET_FLAT_ADAPTIVE, CKV_BUDGET_GIVEN = 0, 1, 2
 CKV_NORM_L1, CKV_NORM_L2 = 0, 1
 CKV_FLAG_WO_SHARED, CKV_FLAG_FORCE_SIMT, CKV_FLAG_WO_GROUP_SUM, CKV_FLAG_PROTECT_WINDOW = 1, 2, 4, 8
 CKV_FLAG_SELECT_MULTIPASS = 32
+CKV_FLAG_SELECT_SINGLE_KERNEL = 16
+CKV_FLAG_SELECT_NO_CLUSTER = 256
 CKV_FLAG_DEBUG_CHECKS = 64
 CKV_FLAG_REQUIRE_TENSOR_CORES = 128
 CKV_EBOUNDS = -7

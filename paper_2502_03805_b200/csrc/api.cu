@@ -57,7 +57,8 @@ int resolve(const criticalkv_desc* d, Dims* o) {
   if (d->reserved != 0 || d->reserved2 != 0) return CKV_EINVAL;
   if (!(d->adaptive_floor >= 0.f && d->adaptive_floor <= 1.f)) return CKV_EINVAL;
   if (d->flags & ~(uint32_t)(CKV_FLAG_WO_SHARED | CKV_FLAG_FORCE_SIMT | CKV_FLAG_WO_GROUP_SUM |
-                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_SELECT_MULTIPASS |
+                             CKV_FLAG_PROTECT_WINDOW | CKV_FLAG_SELECT_MULTIPASS | CKV_FLAG_SELECT_SINGLE_KERNEL |
+                             CKV_FLAG_SELECT_NO_CLUSTER |
                              CKV_FLAG_DEBUG_CHECKS | CKV_FLAG_REQUIRE_TENSOR_CORES))
     return CKV_EINVAL;
   if (d->budget < 0) return CKV_EINVAL;
@@ -316,7 +317,9 @@ int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, const float
   ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets),
                           L.sync_bytes ? (void*)(base + L.sync) : nullptr};
   int launches = 0;
-  const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1};
+  const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1,
+                             (d->flags & CKV_FLAG_SELECT_SINGLE_KERNEL) ? 1 : 0,
+                             (d->flags & CKV_FLAG_SELECT_NO_CLUSTER) ? 0 : 1};
   cudaError_t e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, sd, (cudaStream_t)stream,
                                      &launches, h->status_word, &h->last_select_fused);
   h->launches += launches;
@@ -371,7 +374,7 @@ int criticalkv_allocate_budgets(criticalkv_handle h, const criticalkv_desc* d, c
   DeviceGuard guard(h->device);
   if (!guard.ok) return CKV_ECUDA;
   int launches = 0;
-  cudaError_t e = ckv::launch_allocate_budgets(dd, a, budgets_out, (cudaStream_t)stream, &launches);
+  cudaError_t e = ckv::launch_allocate_budgets(dd, a, budgets_out, h->smem_optin, (cudaStream_t)stream, &launches);
   h->launches += launches;
   return record_cuda(h, e);
 }
@@ -668,7 +671,9 @@ int criticalkv_select_static(criticalkv_handle h, const criticalkv_desc* d, cons
   ckv::SelectWorkspace sw{(float*)(base + L.a), (float*)(base + L.c), (int32_t*)(base + L.budgets),
                           L.sync_bytes ? (void*)(base + L.sync) : nullptr};
   int launches = 0;
-  const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1};
+  const ckv::SelectDevice sd{h->sm_count, h->smem_optin, (d->flags & CKV_FLAG_SELECT_MULTIPASS) ? 0 : 1,
+                             (d->flags & CKV_FLAG_SELECT_SINGLE_KERNEL) ? 1 : 0,
+                             (d->flags & CKV_FLAG_SELECT_NO_CLUSTER) ? 0 : 1};
   e = ckv::launch_select(dd, attn, vnorm, budgets_in, idx, offsets, stage, sw, sd, (cudaStream_t)stream, &launches,
                          h->status_word, &h->last_select_fused);
   h->launches += launches;
@@ -690,7 +695,8 @@ const char* criticalkv_status_string(int s) {
 }
 
 const char* criticalkv_last_cuda_error(criticalkv_handle h) { return h ? h->cuda_error : ""; }
-int criticalkv_last_path(criticalkv_handle h) { return h ? (h->last_path | (h->last_select_fused ? 32 : 0)) : 0; }
+int criticalkv_last_path(criticalkv_handle h) { return h ? (h->last_path | (h->last_select_fused == 1 ? 32 : 0) | (h->last_select_fused == 2 ? 64 : 0)) : 0;
+}
 int64_t criticalkv_launch_count(criticalkv_handle h) { return h ? h->launches : 0; }
 
 }  // extern "C"

@@ -84,15 +84,17 @@ cudaError_t launch_vnorm_l2(const Dims& d, const void* V, const void* WO, float*
 // all-gather): group scores a (and c unless null), and the flattened adaptive allocation over a[nb, Hkv, n].
 cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* vnorm, float* a, float* c,
                                 cudaStream_t st, int* launches);
-cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* budgets_out, cudaStream_t st,
-                                    int* launches);
+cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* budgets_out, int smem_optin,
+                                    cudaStream_t st, int* launches);
 // What the selection launcher needs to know about the device and the caller's wishes.
 struct SelectDevice {
   int sm_count;
   int smem_optin;    // largest dynamic shared memory a CTA may ask for
   int allow_fused;   // 0: always the multi-kernel path (CKV_FLAG_SELECT_MULTIPASS)
+  int prefer_fused;  // 1: the single kernel also for few heads (CKV_FLAG_SELECT_SINGLE_KERNEL)
+  int allow_cluster; // 0: one CTA per head in the multi-kernel path (CKV_FLAG_SELECT_NO_CLUSTER)
 };
-// *fused = 1 when the single-kernel path ran.
+// *fused = 1 when the single-kernel path ran, 2 when the two-stage top-k ran with a cluster per head, else 0.
 cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, const int32_t* budgets_in,
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word, int* fused);
@@ -108,5 +110,11 @@ cudaError_t launch_gather_positions(const Dims& d, const int32_t* pos_in, const 
                                     int32_t* pos_out, int sm_count, int* status_word, cudaStream_t st, int* launches);
 // Dynamic shared memory the multi-kernel two-stage selection needs for a head of n entries.
 size_t two_stage_smem_bytes(int n);
+// The two-stage top-k with a thread-block cluster per (nb slice, KV head), for calls with few heads (a, c: the group
+// scores of launch_group_scores).  cudaErrorNotSupported = not launched (shape or device): use the one-CTA kernel.
+bool two_stage_cluster_applies(const Dims& d, const SelectDevice& dev);
+cudaError_t launch_two_stage_cluster(const Dims& d, const float* a, const float* c, const int32_t* budgets,
+                                     int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectDevice& dev,
+                                     cudaStream_t st, int* launches, int* status_word);
 
 }  // namespace ckv

@@ -195,10 +195,12 @@ struct ClusterShared {
 
 __global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(const float* __restrict__ a,
                                                                               int32_t* __restrict__ budgets, int Hkv,
-                                                                              int n, long long btotal, int floor_b) {
+                                                                              int n, long long btotal, int floor_b,
+                                                                              int cached) {
   namespace cg = cooperative_groups;
   cg::cluster_group cluster = cg::this_cluster();
   __shared__ ClusterShared sh;
+  extern __shared__ __align__(16) uint32_t kcache[];   // cached != 0: the integer keys of this CTA's share
   const int cs = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const int b = blockIdx.x / cs;
   const int heads = Hkv / cs, g0 = rank * heads;
@@ -212,14 +214,22 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(co
   const long long count = (long long)heads * n;
   const float* mine = ab + (long long)g0 * n;
   if (tid == 0) { sh.prefix = 0; sh.krem = (uint32_t)btotal; }
+  // the five walks over this CTA's share read it from shared memory when it fits (a layer at a time), else from L2
+  if (cached) scan_keys(mine, count, [&](long long i, float x) { kcache[i] = order_key(x); });
+  auto each_key = [&](long long first, long long cnt, auto&& f) {
+    if (cached) {
+      for (long long i = tid; i < cnt; i += kSelThreads) f(kcache[first + i]);
+    } else {
+      scan_keys(mine + first, cnt, [&](long long, float x) { f(order_key(x)); });
+    }
+  };
   uint32_t known = 0;
   for (int pass = 0; pass < 4; ++pass) {
     const int shift = 24 - 8 * pass;
     for (int e = tid; e < kSelWarps * 256; e += kSelThreads) (&sh.hist[0][0])[e] = 0;
     __syncthreads();
     const uint32_t prefix = sh.prefix;
-    scan_keys(mine, count, [&](long long, float x) {
-      const uint32_t key = order_key(x);
+    each_key(0, count, [&](uint32_t key) {
       if ((key & known) == prefix) atomicAdd(&sh.hist[warp][(key >> shift) & 255u], 1u);
     });
     __syncthreads();
@@ -266,8 +276,7 @@ __global__ void __launch_bounds__(kSelThreads) adaptive_budget_cluster_kernel(co
   __syncthreads();
   for (int g = 0; g < heads; ++g) {
     uint32_t gt = 0, eq = 0;
-    scan_keys(mine + (long long)g * n, n, [&](long long, float x) {
-      const uint32_t key = order_key(x);
+    each_key((long long)g * n, n, [&](uint32_t key) {
       gt += key > T;
       eq += key == T;
     });
@@ -310,8 +319,8 @@ cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* v
   return cudaGetLastError();
 }
 
-cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* budgets_out, cudaStream_t st,
-                                    int* launches) {
+cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* budgets_out, int smem_optin,
+                                    cudaStream_t st, int* launches) {
   const long long b_adapt = d.budget - d.Hkv * d.floor_b;
   int cs = 8;
   while (cs > 1 && d.Hkv % cs != 0) cs >>= 1;
@@ -320,7 +329,14 @@ cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(d.nb * cs));
     cfg.blockDim = dim3(kSelThreads);
-    cfg.dynamicSmemBytes = 0;
+    const size_t share = (size_t)(d.Hkv / cs) * d.n * sizeof(uint32_t);
+    int cached = share + sizeof(ClusterShared) + 1024 <= (size_t)smem_optin ? 1 : 0;
+    if (cached && cudaFuncSetAttribute(adaptive_budget_cluster_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)share) != cudaSuccess) {
+      (void)cudaGetLastError();
+      cached = 0;
+    }
+    cfg.dynamicSmemBytes = cached ? share : 0;
     cfg.stream = st;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
@@ -330,7 +346,7 @@ cudaError_t launch_allocate_budgets(const Dims& d, const float* a_all, int32_t* 
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     const cudaError_t ec = cudaLaunchKernelEx(&cfg, adaptive_budget_cluster_kernel, a_all, budgets_out, d.Hkv, d.n,
-                                              b_adapt, (int)d.floor_b);
+                                              b_adapt, (int)d.floor_b, cached);
     if (ec == cudaSuccess) launched = true;
     else (void)cudaGetLastError();   // no cluster launch on this device: use the single-CTA kernel
   }
@@ -344,7 +360,9 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
                           int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectWorkspace& ws,
                           const SelectDevice& dev, cudaStream_t st, int* launches, int* status_word, int* fused) {
   *fused = 0;
-  if (dev.allow_fused) {
+  // few heads (a layer at a time): the separate kernels with a cluster of CTAs per head beat one CTA per head
+  const bool few_heads = two_stage_cluster_applies(d, dev);
+  if (dev.allow_fused && (dev.prefer_fused || !few_heads)) {
     // one kernel when the shape allows it; otherwise the three kernels below
     const cudaError_t ef = launch_select_fused(d, attn, vnorm, budgets_in, idx, offsets, stage, ws, dev, st, launches,
                                                status_word);
@@ -358,10 +376,15 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
   if (e != cudaSuccess) return e;
   const int32_t* budgets = nullptr;
   if (d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
-    if ((e = launch_allocate_budgets(d, ws.a, ws.budgets, st, launches)) != cudaSuccess) return e;
+    if ((e = launch_allocate_budgets(d, ws.a, ws.budgets, dev.smem_optin, st, launches)) != cudaSuccess) return e;
     budgets = ws.budgets;
   } else if (d.budget_mode == CKV_BUDGET_GIVEN) {
     budgets = budgets_in;
+  }
+  if (dev.allow_cluster) {
+    e = launch_two_stage_cluster(d, ws.a, ws.c, budgets, idx, offsets, stage, dev, st, launches, status_word);
+    if (e == cudaSuccess) *fused = 2;
+    if (e != cudaErrorNotSupported) return e;
   }
   TwoStageArgs p;
   p.a = ws.a; p.c = ws.c; p.budgets = budgets; p.idx = idx; p.offsets = offsets; p.stage = stage;

@@ -53,7 +53,7 @@ def test_workspace_bytes_are_sane(lib):
     (dict(alpha=1.5), B.CKV_EINVAL), (dict(alpha=-0.1), B.CKV_EINVAL), (dict(eps=-1.0), B.CKV_EINVAL),
     (dict(budget=513), B.CKV_EINVAL), (dict(budget=-1), B.CKV_EINVAL),
     (dict(budget_mode="adaptive", budget=2 * 512 + 1), B.CKV_EINVAL), (dict(budget_mode=9), B.CKV_EINVAL),
-    (dict(norm=3), B.CKV_EINVAL), (dict(adaptive_floor=1.5), B.CKV_EINVAL), (dict(adaptive_floor=-0.1), B.CKV_EINVAL), (dict(flags=1 << 8), B.CKV_EINVAL), (dict(flags=1 << 4), B.CKV_EINVAL),
+    (dict(norm=3), B.CKV_EINVAL), (dict(adaptive_floor=1.5), B.CKV_EINVAL), (dict(adaptive_floor=-0.1), B.CKV_EINVAL), (dict(flags=1 << 9), B.CKV_EINVAL), (dict(flags=1 << 31), B.CKV_EINVAL),
     (dict(k_stride=(0, 0, 63)), B.CKV_EALIGN), (dict(k_stride=(0, 0, 32)), B.CKV_EINVAL),
     (dict(Hq=65, Hkv=65), B.CKV_ENOTSUP),      # more KV heads per slice than the selection kernels handle
 ])

@@ -1,5 +1,6 @@
-"""Steps 3-4 on the GPU: the single-kernel selection and the multi-kernel selection against the oracle on identical float32 scores, where every integer decision must
-agree bit for bit (Algorithm 1, stage 1 / stage 2; Algorithm 2, budget allocation)."""
+"""Steps 3-4 on the GPU: the single-kernel selection, the multi-kernel selection with a cluster of CTAs per head and the
+multi-kernel selection with one CTA per head against the oracle on identical float32 scores, where every integer
+decision must agree bit for bit (Algorithm 1, stage 1 / stage 2; Algorithm 2, budget allocation)."""
 import numpy as np
 import pytest
 import torch
@@ -10,6 +11,16 @@ from oracle import criticalkv_oracle as oc
 pytestmark = pytest.mark.gpu
 
 FUSED_BIT = 32
+CLUSTER_BIT = 64
+
+
+def _paths():
+    """(flags, single kernel ran, cluster kernel ran) of the three implementations of steps 3-4 for a call with few
+    heads; without flags such a call takes the cluster path."""
+    from paper_2502_03805_b200 import binding as B
+    return [(B.CKV_FLAG_SELECT_SINGLE_KERNEL, True, False), (0, False, True),
+            (B.CKV_FLAG_SELECT_MULTIPASS, False, True),
+            (B.CKV_FLAG_SELECT_MULTIPASS | B.CKV_FLAG_SELECT_NO_CLUSTER, False, False)]
 
 
 def _select(P, nu, wl, *, flags=0, budgets_in=None, nb=1, adaptive_floor=0.0):
@@ -25,11 +36,14 @@ def _select(P, nu, wl, *, flags=0, budgets_in=None, nb=1, adaptive_floor=0.0):
     return s.idx.cpu().numpy(), s.offsets.cpu().numpy(), s.stage.cpu().numpy(), s.last_path
 
 
-def _check_against_oracle(P, nu, wl, G, *, flags=0, expect_fused=None, budgets_in=None, adaptive_floor=0.0, **okw):
+def _check_against_oracle(P, nu, wl, G, *, flags=0, expect_fused=None, expect_cluster=None, budgets_in=None,
+                          adaptive_floor=0.0, **okw):
     nb = P.shape[0]
     idx, off, st, path = _select(P, nu, wl, flags=flags, budgets_in=budgets_in, nb=nb, adaptive_floor=adaptive_floor)
     if expect_fused is not None:
         assert bool(path & FUSED_BIT) == expect_fused, path
+    if expect_cluster is not None:
+        assert bool(path & CLUSTER_BIT) == expect_cluster, path
     for b in range(nb):
         ref = oc.select(P[b], nu[b], G=G, budget_mode=wl.budget_mode, budget=wl.budget, alpha=wl.alpha, eps=wl.eps,
                         budgets_in=None if budgets_in is None else budgets_in[b], adaptive_floor=adaptive_floor, **okw)
@@ -72,7 +86,7 @@ SHAPES = [
 
 @pytest.mark.parametrize("case", range(len(SHAPES)))
 @pytest.mark.parametrize("kind", ["plain", "pooled", "ties"])
-def test_single_kernel_and_multi_kernel_selection_match_the_oracle(case, kind):
+def test_all_selection_paths_match_the_oracle(case, kind):
     Hq, Hkv, n, mode, budget, alpha = SHAPES[case]
     if n > 8192 and kind == "ties":
         pytest.skip("the large shape is run on the two realistic score kinds")
@@ -80,10 +94,11 @@ def test_single_kernel_and_multi_kernel_selection_match_the_oracle(case, kind):
     nb = 1 if n > 8192 else 2
     P, nu = _scores(100 + case, nb, Hq, n, ties=kind == "ties", pooled=kind == "pooled")
     wl = small_workload(cfg_id=150 + case, Hq=Hq, Hkv=Hkv, n=n, budget_mode=mode, budget=budget, alpha=alpha)
-    a = _check_against_oracle(P, nu, wl, Hq // Hkv, expect_fused=True)
-    b = _check_against_oracle(P, nu, wl, Hq // Hkv, flags=B.CKV_FLAG_SELECT_MULTIPASS, expect_fused=False)
-    for x, y in zip(a, b):
-        np.testing.assert_array_equal(x, y)
+    outs = [_check_against_oracle(P, nu, wl, Hq // Hkv, flags=f, expect_fused=fu, expect_cluster=cl)
+            for f, fu, cl in _paths()]
+    for other in outs[1:]:
+        for x, y in zip(outs[0], other):
+            np.testing.assert_array_equal(x, y)
 
 
 def test_threshold_bin_larger_than_the_candidate_list_takes_the_full_walk():
@@ -94,10 +109,11 @@ def test_threshold_bin_larger_than_the_candidate_list_takes_the_full_walk():
     P = (r.random((1, Hq, n)).astype(np.float32) ** 4)
     nu = r.integers(1, 3, size=(1, Hq, n)).astype(np.float32)
     P[:] = np.float32(0.25)        # equal attention: c = (0.25 + eps) * nu takes three values per head pair
-    wl = small_workload(cfg_id=170, Hq=Hq, Hkv=Hkv, n=n, budget_mode="uniform", budget=9000)
-    _check_against_oracle(P, nu, wl, 2, expect_fused=True)
-    wl = small_workload(cfg_id=171, Hq=Hq, Hkv=Hkv, n=n, budget_mode="adaptive", budget=17001)
-    _check_against_oracle(P, nu, wl, 2, expect_fused=True)
+    for f, fu, cl in _paths():
+        wl = small_workload(cfg_id=170, Hq=Hq, Hkv=Hkv, n=n, budget_mode="uniform", budget=9000)
+        _check_against_oracle(P, nu, wl, 2, flags=f, expect_fused=fu, expect_cluster=cl)
+        wl = small_workload(cfg_id=171, Hq=Hq, Hkv=Hkv, n=n, budget_mode="adaptive", budget=17001)
+        _check_against_oracle(P, nu, wl, 2, flags=f, expect_fused=fu, expect_cluster=cl)
 
 
 def test_ties_at_the_stage_two_threshold_go_to_the_lower_index():
@@ -109,18 +125,21 @@ def test_ties_at_the_stage_two_threshold_go_to_the_lower_index():
     nu = r.integers(1, 3, size=(1, Hq, n)).astype(np.float32)
     for budget in (700, 1501, 2999):
         wl = small_workload(cfg_id=172, Hq=Hq, Hkv=Hkv, n=n, budget_mode="uniform", budget=budget)
-        _check_against_oracle(P, nu, wl, 1, expect_fused=True)
+        for f, fu, cl in _paths():
+            _check_against_oracle(P, nu, wl, 1, flags=f, expect_fused=fu, expect_cluster=cl)
 
 
 def test_long_heads_and_heads_beyond_the_single_kernel_limit():
     # several words per thread in every walk
     P, nu = _scores(9, 1, 4, 70001)
     wl = small_workload(cfg_id=173, Hq=4, Hkv=2, n=70001, budget_mode="adaptive", budget=14000)
-    _check_against_oracle(P, nu, wl, 2, expect_fused=True)
-    # more than 4096 words per head: left to the multi-kernel path
+    for f, fu, cl in _paths():
+        _check_against_oracle(P, nu, wl, 2, flags=f, expect_fused=fu, expect_cluster=cl)
+    # more than 4096 words per head: beyond the single kernel, which hands the call to the separate kernels
     P, nu = _scores(10, 1, 2, 140003)
     wl = small_workload(cfg_id=177, Hq=2, Hkv=2, n=140003, budget_mode="adaptive", budget=28000)
-    _check_against_oracle(P, nu, wl, 1, expect_fused=False)
+    for f, fu, cl in _paths():
+        _check_against_oracle(P, nu, wl, 1, flags=f, expect_fused=False, expect_cluster=cl or fu)
 
 
 @pytest.mark.parametrize("floor", [0.0, 0.3, 1.0])
@@ -135,13 +154,13 @@ def test_floor_protected_window_and_given_budgets_on_both_paths(floor, protect):
     nu = np.exp(r.standard_normal((1, Hq, n))).astype(np.float32)
     wl = small_workload(cfg_id=174, Hq=Hq, Hkv=Hkv, n=n, w=w, budget_mode="adaptive", budget=budget)
     pf = B.CKV_FLAG_PROTECT_WINDOW if protect else 0
-    for flags, fused in ((pf, True), (pf | B.CKV_FLAG_SELECT_MULTIPASS, False)):
-        _check_against_oracle(P, nu, wl, 2, flags=flags, expect_fused=fused, adaptive_floor=floor,
+    for f, fused, cl in _paths():
+        _check_against_oracle(P, nu, wl, 2, flags=pf | f, expect_fused=fused, expect_cluster=cl, adaptive_floor=floor,
                               protect_w=w if protect else 0)
     wl = small_workload(cfg_id=175, Hq=Hq, Hkv=Hkv, n=n, w=w, budget_mode="given", budget=1200)
     budgets = [[0, 900, 17, 100]]
-    for flags, fused in ((pf, True), (pf | B.CKV_FLAG_SELECT_MULTIPASS, False)):
-        _check_against_oracle(P, nu, wl, 2, flags=flags, expect_fused=fused, budgets_in=budgets,
+    for f, fused, cl in _paths():
+        _check_against_oracle(P, nu, wl, 2, flags=pf | f, expect_fused=fused, expect_cluster=cl, budgets_in=budgets,
                               protect_w=w if protect else 0)
 
 
@@ -152,9 +171,9 @@ def test_group_summed_scores_on_both_paths():
     P = r.random((2, Hq, n)).astype(np.float32) ** 5
     nu = np.exp(r.standard_normal((2, Hkv, n))).astype(np.float32)     # one norm per KV head
     wl = small_workload(cfg_id=176, Hq=Hq, Hkv=Hkv, n=n, budget_mode="adaptive", budget=800)
-    for flags, fused in ((B.CKV_FLAG_WO_GROUP_SUM, True),
-                         (B.CKV_FLAG_WO_GROUP_SUM | B.CKV_FLAG_SELECT_MULTIPASS, False)):
-        _check_against_oracle(P, nu, wl, 4, flags=flags, expect_fused=fused, group_sum=True)
+    for f, fused, cl in _paths():
+        _check_against_oracle(P, nu, wl, 4, flags=B.CKV_FLAG_WO_GROUP_SUM | f, expect_fused=fused, expect_cluster=cl,
+                              group_sum=True)
 
 
 @pytest.mark.parametrize("nb,Hkv,G,mode,budget", [(48, 8, 2, "adaptive", 900), (60, 6, 1, "adaptive", 777),
@@ -165,4 +184,14 @@ def test_more_heads_than_resident_ctas(nb, Hkv, G, mode, budget):
     n = 700
     P, nu = _scores(40 + Hkv, nb, Hkv * G, n, pooled=True)
     wl = small_workload(cfg_id=180 + Hkv, Hq=Hkv * G, Hkv=Hkv, n=n, budget_mode=mode, budget=budget)
-    _check_against_oracle(P, nu, wl, G, expect_fused=True)
+    _check_against_oracle(P, nu, wl, G, expect_fused=True, expect_cluster=False)
+
+
+@pytest.mark.parametrize("nb,Hkv", [(3, 8), (5, 4), (9, 8), (37, 2)])
+def test_cluster_sizes_eight_four_and_two(nb, Hkv):
+    # the number of CTAs per head shrinks as the call has more heads (8 up to 13 heads, 4 up to 27, 2 up to 74)
+    n, G = 5000, 2
+    P, nu = _scores(60 + nb, nb, Hkv * G, n, pooled=True)
+    for mode, budget in (("uniform", 611), ("adaptive", 611 * Hkv)):
+        wl = small_workload(cfg_id=190 + Hkv, Hq=Hkv * G, Hkv=Hkv, n=n, budget_mode=mode, budget=budget)
+        _check_against_oracle(P, nu, wl, G, expect_fused=False, expect_cluster=True)
