@@ -130,21 +130,49 @@ __global__ void __launch_bounds__(kThreads) attn_pass_kernel(AttnArgs a) {
   }
 }
 
-// Merge chunk partials: M = max_c m_c, L = sum_c l_c * exp(m_c - M); store (M, 1 / (w * L)).
-__global__ void attn_combine_kernel(const float* part_m, const float* part_l, float* rowstat, int rows, int nchunks,
-                                    int w) {
-  const int r = blockIdx.x * blockDim.x + threadIdx.x;
-  if (r >= rows) return;
+// Merge chunk partials: M = max_c m_c, L = sum_c l_c * exp(m_c - M); store (M, 1 / (w * L)).  One warp per row, lanes
+// across the partials (a layer at a time a row has up to n / 256 + 2 of them, and a thread walking them one after
+// another took longer than a sweep); the sum runs over each lane's partials in ascending order and then over the
+// lanes in a fixed butterfly, so it is the same on every run.
+constexpr int kCombineThreads = 128;
+__global__ void __launch_bounds__(kCombineThreads) attn_combine_kernel(const float* __restrict__ part_m,
+                                                                       const float* __restrict__ part_l,
+                                                                       float* __restrict__ rowstat, int rows,
+                                                                       int nchunks, int w) {
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.x * (kCombineThreads / 32) + (threadIdx.x >> 5);
+  if (r >= rows) return;   // whole warps leave
   const float* pm = part_m + (long long)r * nchunks;
   const float* pl = part_l + (long long)r * nchunks;
   float M = -INFINITY;
-  for (int c = 0; c < nchunks; ++c) M = fmaxf(M, pm[c]);
-  float L = 0.f;
-  for (int c = 0; c < nchunks; ++c) {
-    if (pm[c] != -INFINITY) L += pl[c] * expf(pm[c] - M);
+  for (int c = lane; c < nchunks; c += 128) {
+    float m4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) m4[q] = c + 32 * q < nchunks ? pm[c + 32 * q] : -INFINITY;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) M = fmaxf(M, m4[q]);
   }
-  rowstat[2 * r] = M;
-  rowstat[2 * r + 1] = 1.0f / (L * (float)w);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  float L = 0.f;
+  for (int c = lane; c < nchunks; c += 128) {
+    float m4[4], l4[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const bool in = c + 32 * q < nchunks;
+      m4[q] = in ? pm[c + 32 * q] : -INFINITY;
+      l4[q] = in ? pl[c + 32 * q] : 0.f;
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+      if (m4[q] != -INFINITY) L += l4[q] * expf(m4[q] - M);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) L += __shfl_xor_sync(0xffffffffu, L, o);
+  if (lane == 0) {
+    rowstat[2 * r] = M;
+    rowstat[2 * r + 1] = 1.0f / (L * (float)w);
+  }
 }
 
 // A CTA pools 4096 consecutive positions of one row from a shared-memory copy (with a halo of (kp-1)/2 on both sides),
@@ -238,7 +266,7 @@ cudaError_t run(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st, 
   dim3 grid(a.nchunks, d.Hq, d.nb);
   k1<<<grid, kThreads, smem, st>>>(a);
   const int rows = d.nb * d.Hq * d.w;
-  attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
+  attn_combine_kernel<<<(rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32), kCombineThreads, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
   k2<<<grid, kThreads, smem, st>>>(a);
   dim3 pgrid((d.n + kPoolTile - 1) / kPoolTile, d.nb * d.Hq);
   launch_maxpool_kernel(pgrid, st, a.abar, attn, d.n, d.kp);
@@ -256,7 +284,7 @@ cudaError_t run_stats(const Dims& d, const AttnArgs& a, cudaStream_t st, int* la
   dim3 grid(a.nchunks, d.Hq, d.nb);
   k1<<<grid, kThreads, smem, st>>>(a);
   const int rows = d.nb * d.Hq * d.w;
-  attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
+  attn_combine_kernel<<<(rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32), kCombineThreads, 0, st>>>(a.part_m, a.part_l, a.rowstat, rows, a.nchunks, d.w);
   *launches += 2;
   return cudaGetLastError();
 }
@@ -279,7 +307,7 @@ cudaError_t run_w(const Dims& d, const AttnArgs& a, float* attn, cudaStream_t st
 
 cudaError_t launch_attn_combine(const float* part_m, const float* part_l, float* rowstat, int rows, int nchunks,
                                 int w, cudaStream_t st) {
-  attn_combine_kernel<<<(rows + 127) / 128, 128, 0, st>>>(part_m, part_l, rowstat, rows, nchunks, w);
+  attn_combine_kernel<<<(rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32), kCombineThreads, 0, st>>>(part_m, part_l, rowstat, rows, nchunks, w);
   return cudaGetLastError();
 }
 
