@@ -111,10 +111,11 @@ cudaError_t launch_gather_positions(const Dims& d, const int32_t* pos_in, const 
 // Dynamic shared memory the multi-kernel two-stage selection needs for a head of n entries.
 size_t two_stage_smem_bytes(int n);
 // The two-stage top-k with a thread-block cluster per (nb slice, KV head), for calls with few heads (a, c: the group
-// scores of launch_group_scores).  cudaErrorNotSupported = not launched (shape or device): use the one-CTA kernel.
+// scores of launch_group_scores, or null: computed in the kernel from attn and vnorm).  cudaErrorNotSupported = not launched (shape or device): use the one-CTA kernel.
 bool two_stage_cluster_applies(const Dims& d, const SelectDevice& dev);
-cudaError_t launch_two_stage_cluster(const Dims& d, const float* a, const float* c, const int32_t* budgets,
-                                     int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectDevice& dev,
-                                     cudaStream_t st, int* launches, int* status_word);
+cudaError_t launch_two_stage_cluster(const Dims& d, const float* attn, const float* vnorm, const float* a,
+                                     const float* c, const int32_t* budgets, int32_t* idx, int32_t* offsets,
+                                     uint8_t* stage, const SelectDevice& dev, cudaStream_t st, int* launches,
+                                     int* status_word);
 
 }  // namespace ckv

@@ -17,40 +17,13 @@
 namespace ckv {
 namespace {
 
-__global__ void group_reduce_kernel(const float* __restrict__ attn, const float* __restrict__ vnorm,
-                                    float* __restrict__ a, float* __restrict__ c, int Hq, int Hkv, int G, int n,
-                                    float eps, int group_sum, int protect_from,
-                                    const int32_t* __restrict__ valid_from) {
+__global__ void group_reduce_kernel(GroupScoreArgs p, float* __restrict__ a, float* __restrict__ c) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
+  if (i >= p.n) return;
   const int g = blockIdx.y, b = blockIdx.z;
-  const long long h0 = (long long)b * Hq + (long long)g * G;
-  const float Gf = (float)G;
   float av, cv;
-  if (group_sum) {
-    // vnorm is per KV head: c = (a + eps) * nu_g
-    float sa = attn[h0 * n + i];
-    for (int q = 1; q < G; ++q) sa = __fadd_rn(sa, attn[(h0 + q) * n + i]);
-    av = __fdiv_rn(sa, Gf);
-    cv = __fmul_rn(__fadd_rn(av, eps), vnorm[((long long)b * Hkv + g) * n + i]);
-  } else {
-    float p = attn[h0 * n + i];
-    float sa = p;
-    float sc = __fmul_rn(__fadd_rn(p, eps), vnorm[h0 * n + i]);
-    for (int q = 1; q < G; ++q) {
-      p = attn[(h0 + q) * n + i];
-      sa = __fadd_rn(sa, p);
-      sc = __fadd_rn(sc, __fmul_rn(__fadd_rn(p, eps), vnorm[(h0 + q) * n + i]));
-    }
-    av = __fdiv_rn(sa, Gf);
-    cv = __fdiv_rn(sc, Gf);
-  }
-  if (i >= protect_from) av = cv = 3.402823466e+38f;  // protected observation window: largest float32
-  // padding in front of a right-aligned head: below every real score (those are >= 0), so it is taken last
-  if (valid_from != nullptr && i < valid_from[b * Hkv + g]) av = cv = -1.0f;
-  if (av == 0.f) av = 0.f;  // -0 and +0 must order alike
-  if (cv == 0.f) cv = 0.f;
-  const long long o = ((long long)b * Hkv + g) * n + i;
+  group_scores_of(p, b, g, i, &av, &cv);
+  const long long o = ((long long)b * p.Hkv + g) * p.n + i;
   a[o] = av;
   if (c != nullptr) c[o] = cv;
 }
@@ -313,8 +286,7 @@ size_t two_stage_smem_bytes(int n) {
 cudaError_t launch_group_scores(const Dims& d, const float* attn, const float* vnorm, float* a, float* c,
                                 cudaStream_t st, int* launches) {
   dim3 rgrid((d.n + 255) / 256, d.Hkv, d.nb);
-  group_reduce_kernel<<<rgrid, 256, 0, st>>>(attn, vnorm, a, c, d.Hq, d.Hkv, d.G, d.n, d.eps, d.group_sum,
-                                             d.protect_window ? d.n - d.w : d.n, d.valid_from);
+  group_reduce_kernel<<<rgrid, 256, 0, st>>>(group_score_args(d, attn, vnorm), a, c);
   *launches += 1;
   return cudaGetLastError();
 }
@@ -372,7 +344,16 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
     }
     if (ef != cudaErrorNotSupported) return ef;
   }
-  cudaError_t e = launch_group_scores(d, attn, vnorm, ws.a, ws.c, st, launches);
+  cudaError_t e;
+  if (few_heads && d.budget_mode != CKV_BUDGET_FLAT_ADAPTIVE) {
+    // uniform or given budgets: the cluster kernel computes the group scores itself
+    e = launch_two_stage_cluster(d, attn, vnorm, nullptr, nullptr,
+                                 d.budget_mode == CKV_BUDGET_GIVEN ? budgets_in : nullptr, idx, offsets, stage, dev, st,
+                                 launches, status_word);
+    if (e == cudaSuccess) *fused = 2;
+    if (e != cudaErrorNotSupported) return e;
+  }
+  e = launch_group_scores(d, attn, vnorm, ws.a, ws.c, st, launches);
   if (e != cudaSuccess) return e;
   const int32_t* budgets = nullptr;
   if (d.budget_mode == CKV_BUDGET_FLAT_ADAPTIVE) {
@@ -382,7 +363,8 @@ cudaError_t launch_select(const Dims& d, const float* attn, const float* vnorm, 
     budgets = budgets_in;
   }
   if (dev.allow_cluster) {
-    e = launch_two_stage_cluster(d, ws.a, ws.c, budgets, idx, offsets, stage, dev, st, launches, status_word);
+    e = launch_two_stage_cluster(d, attn, vnorm, ws.a, ws.c, budgets, idx, offsets, stage, dev, st, launches,
+                                 status_word);
     if (e == cudaSuccess) *fused = 2;
     if (e != cudaErrorNotSupported) return e;
   }

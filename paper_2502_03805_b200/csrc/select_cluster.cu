@@ -3,7 +3,8 @@
 // that a single layer's eight heads occupy 64 SMs instead of 8 (8, 4 or 2 CTAs per head, as many as are resident at once).
 //
 // CTA r of a head's cluster owns the contiguous index range [r * m, (r + 1) * m) and keeps the order-preserving integer
-// keys of a_g and c_g of that range in shared memory for the whole kernel (the scores cross L2 once).  A top-k is a
+// keys of a_g and c_g of that range in shared memory for the whole kernel (the scores cross L2 once; unless the budgets
+// are the flattened adaptive ones, which need a_g of all heads first, the group scores are computed here as well).  A top-k is a
 // radix select in four passes of 8 bits: every CTA histograms its own keys, all CTAs read every peer's histogram
 // through distributed shared memory and so walk the same decisions without any broadcast (two hardware cluster
 // barriers per pass).  Ties go to the lower index: a CTA learns through the same exchange how many entries equal to
@@ -31,6 +32,7 @@ struct HeadShared {
 };
 
 struct ClusterArgs {
+  GroupScoreArgs gs;       // a == nullptr: the group scores are computed here from attn and vnorm
   const float* a;
   const float* c;
   const int32_t* budgets;  // [nb, Hkv] or nullptr for uniform
@@ -191,11 +193,20 @@ __global__ void __launch_bounds__(kSelThreads) two_stage_cluster_kernel(ClusterA
   // this CTA's entries
   const int i0 = rank * m;
   const int cnt = max(0, min(m, n - i0));
-  const float* ag = p.a + ((long long)b * p.Hkv + g) * n + i0;
-  const float* cg_ = p.c + ((long long)b * p.Hkv + g) * n + i0;
-  for (int i = threadIdx.x; i < m; i += kSelThreads) {
-    ka[i] = i < cnt ? order_key(ag[i]) : 0u;
-    kc[i] = i < cnt ? order_key(cg_[i]) : 0u;
+  if (p.a != nullptr) {
+    const float* ag = p.a + ((long long)b * p.Hkv + g) * n + i0;
+    const float* cg_ = p.c + ((long long)b * p.Hkv + g) * n + i0;
+    for (int i = threadIdx.x; i < m; i += kSelThreads) {
+      ka[i] = i < cnt ? order_key(ag[i]) : 0u;
+      kc[i] = i < cnt ? order_key(cg_[i]) : 0u;
+    }
+  } else {
+    for (int i = threadIdx.x; i < m; i += kSelThreads) {
+      float av = 0.f, cv = 0.f;
+      if (i < cnt) group_scores_of(p.gs, b, g, i0 + i, &av, &cv);
+      ka[i] = i < cnt ? order_key(av) : 0u;
+      kc[i] = i < cnt ? order_key(cv) : 0u;
+    }
   }
   __syncthreads();
 
@@ -267,14 +278,16 @@ bool two_stage_cluster_applies(const Dims& d, const SelectDevice& dev) {
 }
 
 // cudaErrorNotSupported: the shape does not fit or the device refuses the cluster launch; nothing has been launched.
-cudaError_t launch_two_stage_cluster(const Dims& d, const float* a, const float* c, const int32_t* budgets,
-                                     int32_t* idx, int32_t* offsets, uint8_t* stage, const SelectDevice& dev,
-                                     cudaStream_t st, int* launches, int* status_word) {
+cudaError_t launch_two_stage_cluster(const Dims& d, const float* attn, const float* vnorm, const float* a,
+                                     const float* c, const int32_t* budgets, int32_t* idx, int32_t* offsets,
+                                     uint8_t* stage, const SelectDevice& dev, cudaStream_t st, int* launches,
+                                     int* status_word) {
   int cs, m;
   size_t dyn;
   if (!cluster_shape(d, dev, &cs, &m, &dyn)) return cudaErrorNotSupported;
   const long long heads = (long long)d.nb * d.Hkv;
   ClusterArgs p;
+  p.gs = group_score_args(d, attn, vnorm);
   p.a = a; p.c = c; p.budgets = budgets; p.idx = idx; p.offsets = offsets; p.stage = stage; p.status = status_word;
   p.Hkv = d.Hkv; p.n = d.n; p.m = m; p.uniform_b = d.budget; p.btot = d.btot; p.alpha = d.alpha;
   p.debug = d.debug_checks;

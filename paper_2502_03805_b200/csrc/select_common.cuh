@@ -16,6 +16,58 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// Group scores of entry i of KV head g in slice b (Algorithm 1: attention and perturbation-aware score of a KV group):
+// a = mean_h attn_h, c = mean_h (attn_h + eps) * vnorm_h over the group's query heads (group_sum: c = (a + eps) * the
+// one norm of the KV head), every operation a separately rounded float32 op in this fixed order: the selection is
+// decided in exactly this arithmetic by every kernel.
+struct GroupScoreArgs {
+  const float* attn;
+  const float* vnorm;
+  const int32_t* valid_from;   // [nb, Hkv] or null
+  int Hq, Hkv, G, n;
+  float eps;
+  int group_sum;
+  int protect_from;            // entries >= protect_from are raised to the largest float32 (n when nothing is protected)
+};
+inline GroupScoreArgs group_score_args(const Dims& d, const float* attn, const float* vnorm) {
+  GroupScoreArgs p;
+  p.attn = attn; p.vnorm = vnorm; p.valid_from = d.valid_from;
+  p.Hq = d.Hq; p.Hkv = d.Hkv; p.G = d.G; p.n = d.n; p.eps = d.eps; p.group_sum = d.group_sum;
+  p.protect_from = d.protect_window ? d.n - d.w : d.n;
+  return p;
+}
+__device__ __forceinline__ void group_scores_of(const GroupScoreArgs& p, int b, int g, int i, float* a_out,
+                                                float* c_out) {
+  const long long n = p.n;
+  const long long h0 = (long long)b * p.Hq + (long long)g * p.G;
+  const float Gf = (float)p.G;
+  float av, cv;
+  if (p.group_sum) {
+    float sa = p.attn[h0 * n + i];
+    for (int q = 1; q < p.G; ++q) sa = __fadd_rn(sa, p.attn[(h0 + q) * n + i]);
+    av = __fdiv_rn(sa, Gf);
+    cv = __fmul_rn(__fadd_rn(av, p.eps), p.vnorm[((long long)b * p.Hkv + g) * n + i]);
+  } else {
+    float x = p.attn[h0 * n + i];
+    float sa = x;
+    float sc = __fmul_rn(__fadd_rn(x, p.eps), p.vnorm[h0 * n + i]);
+    for (int q = 1; q < p.G; ++q) {
+      x = p.attn[(h0 + q) * n + i];
+      sa = __fadd_rn(sa, x);
+      sc = __fadd_rn(sc, __fmul_rn(__fadd_rn(x, p.eps), p.vnorm[(h0 + q) * n + i]));
+    }
+    av = __fdiv_rn(sa, Gf);
+    cv = __fdiv_rn(sc, Gf);
+  }
+  if (i >= p.protect_from) av = cv = 3.402823466e+38f;  // protected observation window: largest float32
+  // padding in front of a right-aligned head: below every real score (those are >= 0), so it is taken last
+  if (p.valid_from != nullptr && i < p.valid_from[b * p.Hkv + g]) av = cv = -1.0f;
+  if (av == 0.f) av = 0.f;  // -0 and +0 must order alike
+  if (cv == 0.f) cv = 0.f;
+  *a_out = av;
+  *c_out = cv;
+}
+
 struct SelectShared {
   uint32_t hist[kSelWarps][256];
   uint32_t total[256];
