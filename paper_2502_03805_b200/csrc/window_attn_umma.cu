@@ -522,17 +522,28 @@ cudaError_t launch_window_attn_umma(const Dims& d, const void* Qw, const void* K
   a.head_groups = (Gi + max_hpg - 1) / max_hpg;
   a.heads_per_group = (Gi + a.head_groups - 1) / a.head_groups;
   a.ntiles = (d.n + kKeyTile - 1) / kKeyTile;
-  // enough work items to fill the machine a few times over, but at least 4 key tiles each so that the partial
-  // statistics (two per item) fit the workspace sized for one partial per 256 keys
+  // Work items: a KV group's key tiles are cut into chunks of tiles_per_item; CTA x takes the items x, x + grid, ...
+  // The sweep lasts as long as the CTA with the most tiles, so the chunk length is chosen to make the last round of
+  // items as full as possible (cost of a candidate = rounds * (tiles per item + about half a tile per item for the Q
+  // reload and the pipeline restart)); at least 4 key tiles per item, so that the partial statistics (two per item)
+  // fit the workspace sized for one partial per 256 keys.
   const long long groups = (long long)d.nb * d.Hkv * a.subgroups;
-  long long want_items = 4LL * sm_count;
-  int tpi = (int)((groups * a.ntiles + want_items - 1) / want_items);
-  if (tpi < 4 * kHalves) tpi = 4 * kHalves;
-  if (tpi > 64) tpi = 64;
+  const int max_stride = (d.n + kAttnChunk - 1) / kAttnChunk + 2;
+  int tpi = 0;
+  long long best_cost = 0;
+  for (int cand = 4 * kHalves; cand <= 64; ++cand) {
+    const long long chunks = (a.ntiles + cand - 1) / cand;
+    if (2 * kHalves * chunks > max_stride) continue;
+    const long long items = groups * chunks;
+    const long long grid_c = items < sm_count ? items : sm_count;
+    const long long rounds = (items + grid_c - 1) / grid_c;
+    const long long cost = rounds * (2 * (long long)(cand < a.ntiles ? cand : a.ntiles) + 1);
+    if (tpi == 0 || cost < best_cost) { tpi = cand; best_cost = cost; }
+  }
+  if (tpi == 0) return cudaErrorNotSupported;   // workspace layout
   a.tiles_per_item = tpi;
   a.chunks_per_bg = (a.ntiles + tpi - 1) / tpi;
   a.part_stride = 2 * kHalves * a.chunks_per_bg;
-  if (a.part_stride > (d.n + kAttnChunk - 1) / kAttnChunk + 2) return cudaErrorNotSupported;  // workspace layout
   a.nitems = groups * a.chunks_per_bg;
   a.scale = d.scale;
   a.c = d.scale * kLog2e;
