@@ -168,6 +168,10 @@ CKV_API int criticalkv_score(criticalkv_handle h, const criticalkv_desc* d, cons
  * (Algorithm 1); ties go to the lower index; idx is ascending inside each head's segment
  * [offsets[g], offsets[g+1]).  stage may be NULL.  With given budgets whose sum is below the capacity the tail of
  * idx is left untouched; budgets outside [0, n] or beyond the capacity are clipped and flagged in the status word.
+ * Three implementations give the same bits: one kernel with a CTA per head (default when nb * Hkv exceeds half the
+ * number of SMs), separate kernels with a thread-block cluster per head (default for fewer heads, i.e. a layer at a
+ * time), separate kernels with a CTA per head (heads too long for the other two); CKV_FLAG_SELECT_* override the
+ * choice and criticalkv_last_path reports it.
  */
 CKV_API int criticalkv_select(criticalkv_handle h, const criticalkv_desc* d, const float* attn, const float* vnorm,
                               const int32_t* budgets_in, int32_t* idx, int32_t* offsets, uint8_t* stage, void* ws,

@@ -44,6 +44,11 @@ def test_workspace_bytes_are_sane(lib):
     assert sb >= 4 * 512 * 4 and tb >= 2 * 2 * 512 * 4
     sb2, tb2 = B.criticalkv_workspace_bytes(_desc(nb=3))
     assert sb2 > sb and tb2 > tb
+    # every documented flag is accepted, alone and together with the others of its group
+    for flags in (B.CKV_FLAG_SELECT_MULTIPASS, B.CKV_FLAG_SELECT_SINGLE_KERNEL, B.CKV_FLAG_SELECT_NO_CLUSTER,
+                  B.CKV_FLAG_SELECT_MULTIPASS | B.CKV_FLAG_SELECT_NO_CLUSTER, B.CKV_FLAG_DEBUG_CHECKS,
+                  B.CKV_FLAG_REQUIRE_TENSOR_CORES, B.CKV_FLAG_PROTECT_WINDOW, B.CKV_FLAG_WO_SHARED):
+        assert B.criticalkv_workspace_bytes(_desc(flags=flags)) == (sb, tb) or flags == B.CKV_FLAG_WO_SHARED
 
 
 @pytest.mark.parametrize("kw,status", [
